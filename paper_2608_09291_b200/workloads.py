@@ -1,0 +1,68 @@
+"""Seeded synthetic inputs (weights, activations, scales) shared by the tests, the bench and
+the oracle checks. Holds none of the method's arithmetic: it only draws random numbers.
+
+The shapes stand in for the LLaMA-2-7B/13B/70B projection matrices the paper's kernel corpus is
+built from (paper Sec. VII-A); masks are Bernoulli, either uniform or with a per-row keep rate.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+ROW_CHUNK = 1024
+_X_STREAM = 10 ** 6
+
+
+def make_weight(M: int, K: int, sparsity: float, seed: int, row_varying: bool = False) -> np.ndarray:
+    """Dense int8 matrix, values uniform on [-8,7] without 0 where kept, 0 where pruned.
+
+    Rows are drawn in chunks of 1024 from ``default_rng([seed, chunk])``: (row-varying only)
+    per-row keep rates ~U(0.3, 0.7), then the keep draws, then the values.
+    """
+    W = np.zeros((M, K), dtype=np.int8)
+    for c, r0 in enumerate(range(0, M, ROW_CHUNK)):
+        rows = min(ROW_CHUNK, M - r0)
+        rng = np.random.default_rng([seed, c])
+        if row_varying:
+            p = rng.uniform(0.3, 0.7, rows)
+        U = rng.random((rows, K))
+        keep = U < (p[:, None] if row_varying else (1.0 - sparsity))
+        v = rng.integers(0, 15, (rows, K))
+        v = np.where(v < 8, v - 8, v - 7).astype(np.int8)
+        W[r0:r0 + rows] = np.where(keep, v, 0)
+    return W
+
+
+def make_x(K: int, N_max: int, seed: int) -> np.ndarray:
+    """Activations, int8 values uniform on [-8,7], token-major (N_max, K)."""
+    rng = np.random.default_rng([seed, _X_STREAM])
+    return rng.integers(-8, 8, (N_max, K)).astype(np.int8)
+
+
+def make_scales(M: int, N_max: int, seed: int):
+    """fp16 per-output-channel weight scales ~U(0.005,0.02) and per-token activation scales
+    ~U(0.01,0.05)."""
+    rng = np.random.default_rng([seed, _X_STREAM + 1])
+    s_w = rng.uniform(0.005, 0.02, M).astype(np.float16)
+    s_x = rng.uniform(0.01, 0.05, N_max).astype(np.float16)
+    return s_w, s_x
+
+
+# The synthetic configurations of the build's target (name -> list of cases).
+def config_cases(name: str):
+    if name == "single":
+        return [dict(M=1024, K=1024, s=0.5, N=[8], seed=0, row_varying=False)]
+    if name == "attn7b":
+        return [dict(M=4096, K=4096, s=s, N=[1, 8, 16, 32], seed=200 + i, row_varying=False)
+                for i, s in enumerate((0.3, 0.5, 0.7))]
+    if name == "ffn7b":
+        return [dict(M=11008, K=4096, s=0.5, N=[1, 8, 32], seed=300, row_varying=True),
+                dict(M=11008, K=4096, s=0.5, N=[1, 8, 32], seed=301, row_varying=True),
+                dict(M=4096, K=11008, s=0.5, N=[1, 8, 32], seed=302, row_varying=True)]
+    if name == "layer13b":
+        shapes = [(5120, 5120)] * 4 + [(13824, 5120)] * 2 + [(5120, 13824)]
+        return [dict(M=m, K=k, s=s, N=[16], seed=400 + 10 * j + i, row_varying=False)
+                for j, s in enumerate((0.3, 0.5, 0.7)) for i, (m, k) in enumerate(shapes)]
+    if name == "ffn70b":
+        return [dict(M=28672, K=8192, s=0.6, N=[1, 4, 8, 16, 32, 64], seed=500, row_varying=False),
+                dict(M=8192, K=28672, s=0.6, N=[1, 4, 8, 16, 32, 64], seed=501, row_varying=False)]
+    raise KeyError(name)
