@@ -1,0 +1,138 @@
+/*
+ * unionsparse.h -- C ABI of the B200 (sm_100a) W4A4 bitmap-sparse SpMM library.
+ *
+ *   Y = W * X,  W: M x K pruned INT4 weights held in a bitmap format (IE-BME, paper Sec. V-A),
+ *               X: K x N dense INT4 activations, INT32 accumulation,
+ *               optional fused dequantisation Y16 = fp16(acc * s_w[m] * s_x[n]).
+ *
+ * Every call returns a us_status; nothing aborts, traps or blocks on the GPU. Pointers are
+ * plain host or device pointers as stated per argument; no framework types cross this ABI.
+ * Unless stated otherwise a call may be made from any host thread, but calls on one handle
+ * must not overlap.
+ */
+#ifndef UNIONSPARSE_H_
+#define UNIONSPARSE_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum us_status {
+    US_OK = 0,
+    US_ERR_INVALID_ARG = 1,   /* NULL pointer, non-positive size, N outside 1..max_N, ...   */
+    US_ERR_VALUE_RANGE = 2,   /* a weight outside [-8, 7]                                   */
+    US_ERR_SHAPE = 3,         /* format parameters that do not divide / do not fill words   */
+    US_ERR_UNSUPPORTED = 4,   /* a valid IE-BME format no kernel of this library implements */
+    US_ERR_ALLOC = 5,         /* host or device allocation failed                           */
+    US_ERR_CUDA = 6,          /* a CUDA runtime call failed (see us_last_error)             */
+    US_ERR_DEVICE_TIMEOUT = 7 /* a bounded wait inside a kernel gave up (no hang, no trap)  */
+} us_status;
+
+/*
+ * IE-BME format parameters (paper Sec. V-A "Area Partitioning"): a local tile of H_L x K_L
+ * weights is split into an R_A x C_A grid of areas; one union-mask bit covers the Q = R_A*C_A
+ * values at the same position of every area. Supported by the kernels: H_L = 16, K_L a multiple
+ * of 128 (default 1024), (R_A, C_A) = (2, 1): one bit covers rows i and i+8 of a 16-row strip.
+ */
+typedef struct us_format {
+    int32_t H_L, K_L, R_A, C_A;
+} us_format;
+
+/* Statistics of an encoded matrix (paper Sec. V-A storage arrays and Eq. 1). */
+typedef struct us_stats {
+    int64_t M, K;                 /* logical shape                                          */
+    int64_t Mp, Kp;               /* shape after zero padding to whole tiles                */
+    int64_t nnz;                  /* true nonzeros                                          */
+    int64_t n_tiles;              /* local tiles (one offset each)                          */
+    int64_t sum_P;                /* sum over tiles of P_t = active union-mask bits         */
+    int64_t bytes_payload;        /* ceil(Q * sum_P / 2): the packed INT4 values            */
+    int64_t bytes_payload_padded; /* payload bytes as stored (lane streams padded per tile) */
+    int64_t bytes_bitmap;         /* union bitmaps                                          */
+    int64_t bytes_offsets;        /* 4 * (n_tiles + 1)                                      */
+    int64_t bytes_total;          /* bytes_payload_padded + bytes_bitmap + bytes_offsets    */
+    double  pmr;                  /* Eq. 1: 0.5 * nnz / (bytes_bitmap + bytes_offsets)      */
+    double  fill;                 /* stored values / (M*K) = Q * sum_P / (M*K)              */
+    us_format fmt;                /* the format in use                                      */
+} us_stats;
+
+typedef struct us_handle us_handle;
+
+/* Flags of us_encode. */
+#define US_ENCODE_HOST_ONLY 1u /* build the format on the host only: no CUDA call is made;
+                                  the handle serves us_get_stats / us_decode, not us_spmm    */
+#define US_ENCODE_SORT_ROWS 2u /* order rows by nonzero count before cutting 16-row strips,
+                                  so that rows of similar density share a strip; the output
+                                  row order of us_spmm is unchanged (folded into the store)  */
+
+/*
+ * Offline encoder (paper Sec. V-A, Fig. 7: dense pruned INT4 -> union bitmaps, per-tile
+ * offsets, packed INT4 values), followed by the upload to the current CUDA device.
+ *   W        host, M x K row-major int8, values in [-8, 7], 0 = pruned. Not retained.
+ *   w_scale  host, M fp16 bit patterns (per-output-channel scales), or NULL when only INT32
+ *            output will be requested. Not retained.
+ *   fmt      NULL selects {16, 1024, 2, 1}.
+ *   max_N    largest N later passed to us_spmm (1..64); sizes the split-K workspace.
+ *   out      receives the handle; it owns every host and device array it allocates.
+ * M, K need not be multiples of the tile: the matrix is zero padded internally.
+ * Errors: INVALID_ARG, VALUE_RANGE, SHAPE, UNSUPPORTED, ALLOC, CUDA. On error *out is NULL.
+ */
+us_status us_encode(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_scale,
+                    const us_format* fmt, int32_t max_N, uint32_t flags, us_handle** out);
+
+/* Pure host read of the statistics, PMR (paper Eq. 1) included. */
+us_status us_get_stats(const us_handle* h, us_stats* out);
+
+/*
+ * Test hook: exact inverse of the encoder, from the handle's host copy of the encoded arrays
+ * (paper Sec. V-A read backwards). W_out: host, M x K int8.
+ */
+us_status us_decode(const us_handle* h, int8_t* W_out);
+
+/*
+ * Test hook: the row order in use. perm_out: host, Mp int32 entries; entry p is the original
+ * row stored at padded position p (strip p/16, row p%16), or -1 for a padding row.
+ */
+us_status us_get_row_order(const us_handle* h, int32_t* perm_out);
+
+/*
+ * The SpMM (paper Alg. 2: W in IE-BME format, dense X -> Y), enqueue-only.
+ *   X        device, N x K token-major packed INT4: byte n*ceil(K/2) + k/2 holds k even in its
+ *            low nibble and k odd in its high nibble, two's complement. 16-byte aligned.
+ *   N        1..max_N.
+ *   x_scale  device, N fp16 per-token scales, or NULL.
+ *   Y        device, token-major N x M: int32 when x_scale is NULL, else fp16
+ *            fp16(acc * w_scale[m] * x_scale[n]) (needs a handle encoded with w_scale).
+ *   stream   a cudaStream_t (NULL = the default stream).
+ * Caller owns X, x_scale and Y. Returns before the kernel completes; device-side failures are
+ * reported by us_last_error. One call per handle may be in flight: the split-K workspace and
+ * arrival counters belong to the handle and are left zeroed by each call.
+ * Errors: INVALID_ARG, UNSUPPORTED (host-only handle), CUDA.
+ */
+us_status us_spmm(us_handle* h, const void* X, int32_t N, const void* x_scale, void* Y,
+                  void* stream);
+
+/*
+ * Synchronises the device, then reports the first failure recorded for this handle: a CUDA
+ * error of an earlier launch (US_ERR_CUDA) or a bounded in-kernel wait that ran out
+ * (US_ERR_DEVICE_TIMEOUT). Clears the record.
+ */
+us_status us_last_error(us_handle* h);
+
+/* Frees device and host memory. NULL is accepted. */
+us_status us_destroy(us_handle* h);
+
+/* Algorithmic bytes one us_spmm call moves: encoded W as stored + X + Y + scales. */
+int64_t us_spmm_bytes(const us_handle* h, int32_t N, int32_t fp16_out);
+
+/* Launch geometry of the next us_spmm(N): CTAs, threads per CTA, dynamic shared memory. */
+us_status us_launch_info(const us_handle* h, int32_t N, int32_t* grid, int32_t* block,
+                         int32_t* smem_bytes);
+
+const char* us_status_string(us_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* UNIONSPARSE_H_ */

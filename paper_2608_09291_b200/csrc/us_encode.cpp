@@ -1,0 +1,239 @@
+// Host encoder / decoder of the lane-stream IE-BME layout (see us_host.h), statistics
+// (paper Sec. V-A storage arrays, Eq. 1) and the CTA schedule. Pure C++: no CUDA here.
+#include <algorithm>
+#include <atomic>
+#include <cstring>
+#include <numeric>
+#include <thread>
+
+#include "us_host.h"
+
+namespace us {
+
+namespace {
+
+int pick_threads(int threads, int64_t work_units)
+{
+    if (threads <= 0) threads = (int)std::thread::hardware_concurrency();
+    if (threads <= 0) threads = 1;
+    if ((int64_t)threads > work_units) threads = (int)std::max<int64_t>(1, work_units);
+    return std::min(threads, 64);
+}
+
+template <class F>
+void parallel_for(int64_t n, int threads, F&& f)
+{
+    threads = pick_threads(threads, n);
+    if (threads == 1) {
+        for (int64_t i = 0; i < n; ++i) f(i, 0);
+        return;
+    }
+    std::vector<std::thread> pool;
+    std::atomic<int64_t> next{0};
+    for (int t = 0; t < threads; ++t)
+        pool.emplace_back([&, t] {
+            for (;;) {
+                int64_t i = next.fetch_add(1);
+                if (i >= n) break;
+                f(i, t);
+            }
+        });
+    for (auto& th : pool) th.join();
+}
+
+}  // namespace
+
+int32_t default_K_L(int64_t M, int64_t K)
+{
+    // Large tiles keep the per-tile padding of the lane streams small; small matrices get
+    // smaller tiles so that every warp of a 148-SM part still finds work.
+    const int64_t strips = (M + 15) / 16;
+    for (int32_t kl : {1024, 512, 256}) {
+        int64_t items = strips * ((K + kl - 1) / kl);
+        if (items >= 148 * 16 || kl == 256) return kl;
+    }
+    return 256;
+}
+
+us_status encode_host(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_scale,
+                      const us_format& fmt, uint32_t flags, int threads, HostMatrix* out)
+{
+    if (!W || !out || M <= 0 || K <= 0) return US_ERR_INVALID_ARG;
+    if (fmt.H_L <= 0 || fmt.K_L <= 0 || fmt.R_A <= 0 || fmt.C_A <= 0) return US_ERR_SHAPE;
+    if (fmt.H_L % fmt.R_A || fmt.K_L % fmt.C_A) return US_ERR_SHAPE;
+    if (((int64_t)(fmt.H_L / fmt.R_A) * (fmt.K_L / fmt.C_A)) % 64) return US_ERR_SHAPE;
+    if (fmt.H_L != 16 || fmt.R_A != 2 || fmt.C_A != 1 || fmt.K_L % 128 || fmt.K_L > 8192)
+        return US_ERR_UNSUPPORTED;
+
+    HostMatrix& h = *out;
+    h = HostMatrix();
+    h.M = M; h.K = K; h.fmt = fmt;
+    h.Mp = (M + 15) / 16 * 16;
+    h.Kp = (K + fmt.K_L - 1) / fmt.K_L * fmt.K_L;
+    h.nkb = fmt.K_L / 32;
+    h.mask_rows = h.nkb / 4;
+    h.n_strips = h.Mp / 16;
+    h.n_segs = h.Kp / fmt.K_L;
+    h.n_items = h.n_strips * h.n_segs;
+    if (w_scale) h.w_scale.assign(w_scale, w_scale + M);
+
+    // ---- row order -----------------------------------------------------------------------
+    h.row_order.assign(h.Mp, -1);
+    std::atomic<int> bad{0};
+    if (flags & US_ENCODE_SORT_ROWS) {
+        std::vector<int64_t> cnt(M, 0);
+        parallel_for(M, threads, [&](int64_t r, int) {
+            const int8_t* p = W + r * K;
+            int64_t c = 0;
+            for (int64_t k = 0; k < K; ++k) c += p[k] != 0;
+            cnt[r] = c;
+        });
+        std::vector<int32_t> idx(M);
+        std::iota(idx.begin(), idx.end(), 0);
+        std::stable_sort(idx.begin(), idx.end(), [&](int32_t a, int32_t b) { return cnt[a] < cnt[b]; });
+        std::copy(idx.begin(), idx.end(), h.row_order.begin());
+    } else {
+        std::iota(h.row_order.begin(), h.row_order.begin() + M, 0);
+    }
+
+    // ---- build every tile blob (parallel over strips) ------------------------------------
+    const int K_L = fmt.K_L, nkb = h.nkb, mask_rows = h.mask_rows;
+    const int64_t mask_bytes = (int64_t)mask_rows * 128;
+    std::vector<std::vector<uint8_t>> blobs(h.n_items);
+    std::atomic<int64_t> nnz{0}, sum_P{0};
+
+    parallel_for(h.n_strips, threads, [&](int64_t rb, int) {
+        const int8_t* rows[16];
+        for (int r = 0; r < 16; ++r) {
+            int32_t o = h.row_order[rb * 16 + r];
+            rows[r] = o < 0 ? nullptr : W + (int64_t)o * K;
+        }
+        std::vector<uint8_t> stream((size_t)32 * nkb * 8);  // lane-major payload bytes
+        std::vector<uint8_t> mask((size_t)32 * nkb);        // lane-major mask bytes
+        int len[32];
+        int64_t my_nnz = 0, my_P = 0;
+        for (int64_t sg = 0; sg < h.n_segs; ++sg) {
+            const int64_t k0 = sg * K_L;
+            std::fill(mask.begin(), mask.end(), 0);
+            std::fill(len, len + 32, 0);
+            for (int g = 0; g < 8; ++g) {
+                const int8_t* pa = rows[g];
+                const int8_t* pb = rows[g + 8];
+                const int64_t kend = std::min<int64_t>(K, k0 + K_L);
+                for (int64_t k = k0; k < kend; ++k) {
+                    int lo = pa ? pa[k] : 0, hi = pb ? pb[k] : 0;
+                    if (!(lo | hi)) continue;
+                    if (lo < -8 || lo > 7 || hi < -8 || hi > 7) { bad.store(1); continue; }
+                    my_nnz += (lo != 0) + (hi != 0);
+                    const int kk = (int)(k - k0), kb = kk >> 5, t = (kk >> 3) & 3, j = kk & 7;
+                    const int lane = 4 * g + t;
+                    mask[(size_t)lane * nkb + kb] |= (uint8_t)(1u << j);
+                    stream[(size_t)lane * nkb * 8 + len[lane]++] =
+                        (uint8_t)(((hi & 0xF) << 4) | ((lo + 8) & 0xF));
+                }
+            }
+            int maxlen = 0;
+            for (int l = 0; l < 32; ++l) { maxlen = std::max(maxlen, len[l]); my_P += len[l]; }
+            const int J = (maxlen + 3) / 4;
+            std::vector<uint8_t>& b = blobs[sg * h.n_strips + rb];
+            b.assign((size_t)mask_bytes + (size_t)J * 128, 0);
+            for (int l = 0; l < 32; ++l) {
+                for (int w = 0; w < mask_rows; ++w)
+                    std::memcpy(&b[(size_t)w * 128 + l * 4], &mask[(size_t)l * nkb + 4 * w], 4);
+                const uint8_t* s = &stream[(size_t)l * nkb * 8];
+                for (int i = 0; i < len[l]; ++i)
+                    b[(size_t)mask_bytes + (size_t)(i >> 2) * 128 + l * 4 + (i & 3)] = s[i];
+            }
+        }
+        nnz += my_nnz;
+        sum_P += my_P;
+    });
+    if (bad.load()) { h = HostMatrix(); return US_ERR_VALUE_RANGE; }
+
+    // ---- offsets and the contiguous blob -------------------------------------------------
+    h.item_off.assign(h.n_items + 1, 0);
+    uint64_t off16 = 0;
+    for (int64_t t = 0; t < h.n_items; ++t) {
+        h.item_off[t] = (uint32_t)off16;
+        off16 += blobs[t].size() / 16;
+        h.max_item_bytes = std::max<uint32_t>(h.max_item_bytes, (uint32_t)blobs[t].size());
+        if (off16 > 0xFFFFFFFFull) { h = HostMatrix(); return US_ERR_ALLOC; }
+    }
+    h.item_off[h.n_items] = (uint32_t)off16;
+    try {
+        h.blob.assign((size_t)off16 * 16, 0);
+    } catch (...) {
+        h = HostMatrix();
+        return US_ERR_ALLOC;
+    }
+    parallel_for(h.n_items, threads, [&](int64_t t, int) {
+        std::memcpy(h.blob.data() + (size_t)h.item_off[t] * 16, blobs[t].data(), blobs[t].size());
+        std::vector<uint8_t>().swap(blobs[t]);
+    });
+    h.nnz = nnz.load();
+    h.sum_P = sum_P.load();
+    h.bytes_payload_padded = (int64_t)h.blob.size() - h.n_items * mask_bytes;
+    return US_OK;
+}
+
+void decode_host(const HostMatrix& h, int8_t* W_out)
+{
+    std::memset(W_out, 0, (size_t)(h.M * h.K));
+    const int nkb = h.nkb, mask_rows = h.mask_rows, K_L = h.fmt.K_L;
+    for (int64_t t = 0; t < h.n_items; ++t) {
+        const int64_t sg = t / h.n_strips, rb = t % h.n_strips;
+        const uint8_t* b = h.blob.data() + (size_t)h.item_off[t] * 16;
+        const uint8_t* pay = b + (size_t)mask_rows * 128;
+        for (int lane = 0; lane < 32; ++lane) {
+            const int g = lane >> 2, tt = lane & 3;
+            const int32_t ra = h.row_order[rb * 16 + g], rbw = h.row_order[rb * 16 + g + 8];
+            int pos = 0;  // byte position in the lane's stream
+            for (int kb = 0; kb < nkb; ++kb) {
+                const uint8_t m = b[(size_t)(kb >> 2) * 128 + lane * 4 + (kb & 3)];
+                for (int j = 0; j < 8; ++j) {
+                    if (!((m >> j) & 1)) continue;
+                    const uint8_t v = pay[(size_t)(pos >> 2) * 128 + lane * 4 + (pos & 3)];
+                    ++pos;
+                    const int64_t k = sg * K_L + 32 * kb + 8 * tt + j;
+                    if (k >= h.K) continue;
+                    const int lo = (int)(v & 0xF) - 8;
+                    const int hi = (v >> 4) >= 8 ? (int)(v >> 4) - 16 : (int)(v >> 4);
+                    if (ra >= 0) W_out[(int64_t)ra * h.K + k] = (int8_t)lo;
+                    if (rbw >= 0) W_out[(int64_t)rbw * h.K + k] = (int8_t)hi;
+                }
+            }
+        }
+    }
+}
+
+void fill_stats(const HostMatrix& h, us_stats* st)
+{
+    const int Q = h.fmt.R_A * h.fmt.C_A;
+    st->M = h.M; st->K = h.K; st->Mp = h.Mp; st->Kp = h.Kp;
+    st->nnz = h.nnz;
+    st->n_tiles = h.n_items;
+    st->sum_P = h.sum_P;
+    st->bytes_payload = ((int64_t)Q * h.sum_P + 1) / 2;
+    st->bytes_payload_padded = h.bytes_payload_padded;
+    st->bytes_bitmap = h.n_items * (int64_t)h.mask_rows * 128;
+    st->bytes_offsets = 4 * (h.n_items + 1);
+    st->bytes_total = st->bytes_payload_padded + st->bytes_bitmap + st->bytes_offsets;
+    st->pmr = 0.5 * (double)h.nnz / (double)(st->bytes_bitmap + st->bytes_offsets);
+    st->fill = (double)Q * (double)h.sum_P / ((double)h.M * (double)h.K);
+    st->fmt = h.fmt;
+}
+
+void make_schedule(const HostMatrix& h, int n_cta, std::vector<uint32_t>* begin)
+{
+    begin->assign((size_t)n_cta + 1, 0);
+    const uint64_t total = h.item_off[h.n_items];
+    int64_t t = 0;
+    for (int c = 0; c <= n_cta; ++c) {
+        const uint64_t target = total * (uint64_t)c / (uint64_t)n_cta;
+        while (t < h.n_items && h.item_off[t] < target) ++t;
+        (*begin)[c] = (uint32_t)t;
+    }
+    (*begin)[n_cta] = (uint32_t)h.n_items;
+}
+
+}  // namespace us

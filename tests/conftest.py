@@ -16,3 +16,12 @@ def pytest_configure(config):
 @pytest.fixture(scope="session")
 def golden_dir():
     return ROOT / "tests" / "golden"
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_libraries():
+    """Compile the CUDA library (nvcc cross-compiles without a GPU) and the C oracle once."""
+    from paper_2608_09291_b200 import build as libbuild
+    import oracle
+    libbuild.build()
+    oracle.build()
