@@ -282,6 +282,8 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
             const uint32_t o0 = p.item_off[it], o1 = p.item_off[it + 1];
             const uint32_t bytes = (o1 - o0) * 16u;
             const uint32_t bar = smem_u32(&bars[warp * STAGES + s]);
+            // the warp's earlier generic-proxy reads of this slot are ordered before the refill
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             mbar_expect_tx(bar, bytes);
             bulk_g2s(smem_u32(my_ring + (size_t)s * p.slot_bytes), p.blob + (size_t)o0 * 16u, bytes, bar);
         }
