@@ -1,0 +1,476 @@
+#!/usr/bin/env python
+"""Benchmark of the W4A4 bitmap-sparse SpMM (one JSON line on stdout).
+
+Workload of the headline line: LLaMA-2-7B-shaped attention projections, W 4096x4096 INT4 at 50 %
+uniform sparsity, X 4096xN INT4 with N = 8, fused fp16 dequant output. One step = one SpMM on each
+of R distinct encoded weight buffers (R * bytes > 3x the L2 size, so every launch streams its
+weights from HBM). The sweep over sparsity {30, 50, 70 %} x N {1, 8, 16, 32} and the 70B-shaped
+FFN (28672x8192, 60 %) N sweep are reported in the same line under "sweep".
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-sweep]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+METRIC = "w4a4_spmm_achieved_hbm_gbs"
+UNIT = "GB/s"
+HEAD = dict(M=4096, K=4096, s=0.5, N=8, seed=201)
+CONTRACT_PEAK_GBS = 8000.0
+L2_BYTES_FALLBACK = 126 * 1024 * 1024
+
+
+def algorithmic_bytes(stats: dict, N: int, fp16: bool) -> int:
+    """What the method must move once per call: packed INT4 values of the active union-mask
+    positions, union bitmaps, per-tile offsets, X, Y and (fp16 output) the two scale vectors.
+    Padding of the stored payload is NOT counted: it shows up as traffic above this figure."""
+    M, K = stats["M"], stats["K"]
+    w = stats["bytes_payload"] + stats["bytes_bitmap"] + stats["bytes_offsets"]
+    return w + N * ((K + 1) // 2) + N * M * (2 if fp16 else 4) + (2 * (M + N) if fp16 else 0)
+
+
+def measured_peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        d = json.loads(p.read_text())
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and clock-event reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period: float = 0.02):
+        super().__init__(daemon=True)
+        self.period, self.samples, self.reasons, self.max_mhz = period, [], set(), None
+        self._stop_evt = threading.Event()
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.dev = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.dev, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def sample(self):
+        if self.nv is None:
+            return
+        nv = self.nv
+        try:
+            self.samples.append(nv.nvmlDeviceGetClockInfo(self.dev, nv.NVML_CLOCK_SM))
+            r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.dev)
+            names = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "sw_thermal_slowdown": 0x20,
+                     "hw_thermal_slowdown": 0x40, "hw_power_brake_slowdown": 0x80,
+                     "sync_boost": 0x10, "applications_clocks_setting": 0x2}
+            for k, bit in names.items():
+                if r & bit:
+                    self.reasons.add(k)
+        except Exception:
+            pass
+
+    def run(self):
+        while not self._stop_evt.is_set():
+            self.sample()
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def visible_device_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# ------------------------------------------------------------------------------------------------
+def reference_arm(args, rank: int):
+    """The CPU oracle, as it stands, timed on the host cores (the reference of this build)."""
+    if rank != 0:
+        return
+    import oracle
+    from paper_2608_09291_b200 import workloads
+    oracle.build()
+    W = workloads.make_weight(HEAD["M"], HEAD["K"], HEAD["s"], HEAD["seed"])
+    X = workloads.make_x(HEAD["K"], 32, HEAD["seed"])[: HEAD["N"]]
+    s_w, s_x = workloads.make_scales(HEAD["M"], 32, HEAD["seed"])
+    st = oracle.encode(W, 16, 1024, 2, 1)["stats"]
+    stats = dict(M=HEAD["M"], K=HEAD["K"], bytes_payload=st["bytes_payload"],
+                 bytes_bitmap=st["bytes_bitmap"], bytes_offsets=st["bytes_offsets"])
+    per_call = algorithmic_bytes(stats, HEAD["N"], True)
+    calls_per_step = 2
+
+    def step():
+        for _ in range(calls_per_step):
+            oracle.dequant(oracle.spmm_dense(W, X), s_w, s_x[: HEAD["N"]])
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    value = per_call * calls_per_step * args.steps / dt / 1e9
+    sample = (f"{calls_per_step} oracle SpMMs (naive masked-dense INT32 GEMM + fp64 dequant) of the "
+              f"4096x4096 s=0.5 N=8 case per step")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32",
+        "data": "synthetic",
+        "config": {"workload": "llama2-7b attention projection 4096x4096 INT4, 50% sparsity, N=8, fp16 dequant",
+                   "flush": "n/a (CPU)"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+# ------------------------------------------------------------------------------------------------
+class Case:
+    """R replicas of one encoded weight plus device inputs; a 'pass' = one SpMM per replica."""
+
+    def __init__(self, binding, torch, W, s_w, X, s_x, N_max, replicas, fmt=None, flags=0):
+        self.torch, self.b = torch, binding
+        self.sw = [binding.SparseWeight(W, s_w, fmt=fmt, max_N=N_max, flags=flags) for _ in range(replicas)]
+        self.stats = self.sw[0].stats
+        self.Xh = torch.from_numpy(binding.pack_int4(X)).pin_memory()
+        self.Xd = self.Xh.cuda()
+        self.sxd = torch.from_numpy(s_x.copy()).cuda() if s_x is not None else None
+        self.M, self.K = W.shape
+        self.Y16 = torch.empty((N_max, self.M), dtype=torch.float16, device="cuda")
+        self.Y32 = torch.empty((N_max, self.M), dtype=torch.int32, device="cuda")
+
+    def enqueue_pass(self, N, fp16):
+        xs = self.sxd if fp16 else None
+        out = self.Y16 if fp16 else self.Y32
+        for sw in self.sw:
+            sw.spmm(self.Xd, N, xs, out=out[:N])
+
+    def graph(self, N, fp16):
+        torch = self.torch
+        g = torch.cuda.CUDAGraph()
+        s = torch.cuda.Stream()
+        s.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(s):
+            self.enqueue_pass(N, fp16)          # warm-up outside capture
+        torch.cuda.current_stream().wait_stream(s)
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g):
+            self.enqueue_pass(N, fp16)
+        return g
+
+    def time_passes(self, N, fp16, passes, warmup):
+        """Median-free plain timing: total device time of `passes` graph replays / launches."""
+        torch = self.torch
+        g = self.graph(N, fp16)
+        for _ in range(warmup):
+            g.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(passes):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        for sw in self.sw:
+            sw.check()
+        return e0.elapsed_time(e1) * 1e-3 / (passes * len(self.sw))   # seconds per launch
+
+    def close(self):
+        for sw in self.sw:
+            sw.close()
+
+
+def replicas_for(stats, l2_bytes):
+    return max(3, int(np.ceil(3.2 * l2_bytes / max(1, stats_bytes(stats)))))
+
+
+def stats_bytes(stats):
+    return stats["bytes_total"]
+
+
+def run_ours(args, rank: int, local_rank: int, world: int):
+    import torch
+    from paper_2608_09291_b200 import build as libbuild
+    if rank == 0:
+        libbuild.build()
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    else:
+        dist = None
+        torch.cuda.set_device(local_rank)
+    from paper_2608_09291_b200 import binding, workloads
+
+    l2 = torch.cuda.get_device_properties(local_rank).L2_cache_size or L2_BYTES_FALLBACK
+    peak_gbs, peak_kind = measured_peaks()
+
+    # ---- headline case -----------------------------------------------------------------------
+    W = workloads.make_weight(HEAD["M"], HEAD["K"], HEAD["s"], HEAD["seed"])
+    Xall = workloads.make_x(HEAD["K"], 32, HEAD["seed"])
+    s_w, s_x = workloads.make_scales(HEAD["M"], 32, HEAD["seed"])
+    probe = binding.us_encode(W, s_w, None, 32, binding.US_ENCODE_HOST_ONLY)
+    pstats = binding.us_get_stats(probe)
+    binding.us_destroy(probe)
+    R = replicas_for(pstats, l2)
+    head = Case(binding, torch, W, s_w, Xall, s_x, 32, R)
+    N = HEAD["N"]
+    alg = algorithmic_bytes(head.stats, N, True)
+    g = head.graph(N, True)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        g.replay()
+    barrier()
+    sampler = ClockSampler(visible_device_index(local_rank))
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        g.replay()
+    e1.record()
+    sampler.sample()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    barrier()
+    for sw in head.sw:
+        sw.check()
+    dt = e0.elapsed_time(e1) * 1e-3
+    if dist is not None:
+        t = torch.tensor([dt], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dt = float(t.item())
+    launches = args.steps * R
+    per_launch = dt / launches
+    value = alg * launches * world / dt / 1e9
+
+    # ---- end to end: host buffers, H2D of X and scales, D2H of Y inside the timed region --------
+    Xh = head.Xh[:N].clone().pin_memory()
+    sxh = torch.from_numpy(s_x[:N].copy()).pin_memory()
+    Yh = torch.empty((N, HEAD["M"]), dtype=torch.float16).pin_memory()
+    Xd = torch.empty_like(Xh, device="cuda")
+    sxd = torch.empty_like(sxh, device="cuda")
+    Yd = torch.empty((N, HEAD["M"]), dtype=torch.float16, device="cuda")
+
+    def e2e_step():
+        for sw in head.sw:
+            Xd.copy_(Xh, non_blocking=True)
+            sxd.copy_(sxh, non_blocking=True)
+            sw.spmm(Xd, N, sxd, out=Yd)
+            Yh.copy_(Yd, non_blocking=True)
+        torch.cuda.synchronize()
+
+    for _ in range(3):
+        e2e_step()
+    e2e_steps = max(3, min(args.steps, 50))
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    t_e2e = time.perf_counter() - t0
+    if dist is not None:
+        t = torch.tensor([t_e2e], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        t_e2e = float(t.item())
+    e2e_value = alg * R * e2e_steps * world / t_e2e / 1e9
+    h2d = R * (Xh.numel() + sxh.numel() * 2)
+    d2h = R * Yh.numel() * 2
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+        "config": {
+            "workload": "llama2-7b attention projection 4096x4096 INT4, 50% uniform sparsity, N=8, "
+                        "fused fp16 dequant; one step = one SpMM on each of R distinct weight buffers",
+            "replicas_per_step": R, "format": list(head.stats["fmt"]),
+            "flush": f"inputs larger than L2: {R} x {head.stats['bytes_total']} B of weights rotate "
+                     f"through a {l2} B L2",
+            "launch": "CUDA graph of one step, replayed",
+            "parallelism": "replicas only" if world > 1 else "1 gpu",
+        },
+        "us_per_spmm": per_launch * 1e6,
+        "dense_equiv_tops": 2.0 * HEAD["M"] * HEAD["K"] * N / per_launch / 1e12,
+        "pct_of_8tbs": 100.0 * (alg / per_launch / 1e9) / CONTRACT_PEAK_GBS,
+        "clocks": clocks,
+        "gpu_launches": launches,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps},
+        "roofline": {"bound": "hbm", "achieved": alg / per_launch / 1e9, "peak": peak_gbs,
+                     "unit": "GB/s", "frac": alg / per_launch / 1e9 / peak_gbs, "peak_kind": peak_kind,
+                     "traffic": TRAFFIC_BYTES_PER_LAUNCH, "algorithmic_bytes": alg,
+                     "stored_bytes": binding.us_spmm_bytes(head.sw[0].handle, N, True),
+                     "kernel": "us_spmm_kernel<1,2> on 4096x4096 s=0.5 N=8"},
+        "stats": {k: head.stats[k] for k in ("nnz", "sum_P", "bytes_payload", "bytes_payload_padded",
+                                             "bytes_bitmap", "bytes_offsets", "pmr", "fill")},
+    }
+    head.close()
+
+    if rank == 0 and not args.no_sweep:
+        out["sweep"] = sweep(binding, torch, workloads, l2, peak_gbs)
+    if rank == 0:
+        out["cpu_baseline"] = cpu_baseline(W, Xall[:N], s_w, s_x[:N], pstats)
+        print(json.dumps(out))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+# Measured DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the
+# headline kernel, from the ncu capture summarised under profiles/; None until captured.
+TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def sweep(binding, torch, workloads, l2, peak_gbs):
+    rows = []
+
+    def run_case(name, M, K, s, seed, Ns, fp16, row_varying=False, flags=0):
+        W = workloads.make_weight(M, K, s, seed, row_varying)
+        Nmax = max(Ns)
+        X = workloads.make_x(K, Nmax, seed)
+        s_w, s_x = workloads.make_scales(M, Nmax, seed)
+        probe = binding.us_encode(W, None, None, Nmax, binding.US_ENCODE_HOST_ONLY | flags)
+        st = binding.us_get_stats(probe)
+        binding.us_destroy(probe)
+        R = replicas_for(st, l2)
+        case = Case(binding, torch, W, s_w, X, s_x, Nmax, R, flags=flags)
+        for N in Ns:
+            passes = max(3, int(2e-2 / max(1e-6, 3e-6 * R)))
+            t = case.time_passes(N, fp16, passes=min(passes, 200), warmup=3)
+            alg = algorithmic_bytes(case.stats, N, fp16)
+            rows.append({"case": name, "M": M, "K": K, "sparsity": s, "N": N, "out": "fp16" if fp16 else "int32",
+                         "us": t * 1e6, "alg_bytes": alg, "stored_bytes": binding.us_spmm_bytes(case.sw[0].handle, N, fp16),
+                         "gbs": alg / t / 1e9, "pct_of_8tbs": 100 * alg / t / 1e9 / CONTRACT_PEAK_GBS,
+                         "frac_of_measured": alg / t / 1e9 / peak_gbs,
+                         "dense_equiv_tops": 2.0 * M * K * N / t / 1e12, "replicas": R,
+                         "pmr": case.stats["pmr"]})
+        case.close()
+        del case
+        torch.cuda.empty_cache()
+
+    for i, s in enumerate((0.3, 0.5, 0.7)):
+        run_case("attn7b", 4096, 4096, s, 200 + i, [1, 8, 16, 32], True)
+    run_case("ffn7b_up", 11008, 4096, 0.5, 300, [8], True, row_varying=True, flags=binding.US_ENCODE_SORT_ROWS)
+    run_case("ffn70b_up", 28672, 8192, 0.6, 500, [1, 4, 8, 16, 32, 64], False)
+    return rows
+
+
+def cpu_baseline(W, X, s_w, s_x, stats):
+    import oracle
+    oracle.build()
+    N = X.shape[0]
+    per_call = algorithmic_bytes(stats, N, True)
+    oracle.dequant(oracle.spmm_dense(W, X), s_w, s_x)
+    calls, t0 = 0, time.perf_counter()
+    while time.perf_counter() - t0 < 10.0 or calls < 3:
+        oracle.dequant(oracle.spmm_dense(W, X), s_w, s_x)
+        calls += 1
+    dt = time.perf_counter() - t0
+    return {"value": per_call * calls / dt / 1e9, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{calls} calls of the oracle (naive masked-dense INT32 GEMM, OpenMP over rows, "
+                      f"+ fp64 dequant) on the 4096x4096 s=0.5 N=8 case, {dt:.1f} s",
+            "ms_per_spmm": dt / calls * 1e3}
+
+
+def run_only(args):
+    import torch
+    from paper_2608_09291_b200 import build as libbuild
+    libbuild.build()
+    from paper_2608_09291_b200 import binding, workloads
+    f = args.only.split(",")
+    M, K, s, N = int(f[0]), int(f[1]), float(f[2]), int(f[3])
+    fp16 = len(f) > 4 and f[4] == "fp16"
+    fmt = (16, int(f[5]), 2, 1) if len(f) > 5 else None
+    torch.cuda.set_device(0)
+    l2 = torch.cuda.get_device_properties(0).L2_cache_size or L2_BYTES_FALLBACK
+    W = workloads.make_weight(M, K, s, seed=1)
+    X = workloads.make_x(K, N, seed=1)
+    s_w, s_x = workloads.make_scales(M, N, seed=1)
+    probe = binding.us_encode(W, None, fmt, N, binding.US_ENCODE_HOST_ONLY)
+    st = binding.us_get_stats(probe)
+    binding.us_destroy(probe)
+    case = Case(binding, torch, W, s_w, X, s_x, N, replicas_for(st, l2), fmt=fmt)
+    for _ in range(max(1, args.warmup)):
+        case.enqueue_pass(N, fp16)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        case.enqueue_pass(N, fp16)
+    e1.record()
+    torch.cuda.synchronize()
+    for sw in case.sw:
+        sw.check()
+    t = e0.elapsed_time(e1) * 1e-3 / (args.steps * len(case.sw))
+    alg = algorithmic_bytes(case.stats, N, fp16)
+    # one more pass with the kernel's stage timers on (not part of the timing above)
+    for sw in case.sw:
+        binding.us_stage_timers(sw.handle, 1)
+    case.enqueue_pass(N, fp16)
+    torch.cuda.synchronize()
+    tm = {}
+    for sw in case.sw:
+        for k, v in binding.us_stage_timers(sw.handle, 0, read=True).items():
+            tm[k] = tm.get(k, 0) + v
+    timers = {k: (v / tm["warps"] if k != "warps" else v / len(case.sw)) for k, v in tm.items()}
+    print(json.dumps({"only": args.only, "us_per_launch_stream_order": t * 1e6, "alg_bytes": alg,
+                      "stored_bytes": binding.us_spmm_bytes(case.sw[0].handle, N, fp16),
+                      "gbs": alg / t / 1e9, "replicas": len(case.sw), "format": list(case.stats["fmt"]),
+                      "launch": binding.us_launch_info(case.sw[0].handle, N),
+                      "stage_cycles_per_warp": timers}))
+    case.close()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--only", default=None, metavar="M,K,s,N[,int32|fp16[,K_L]]",
+                    help="time one case only (a few launches, no graph): the small run used for ncu captures")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        reference_arm(args, rank)
+        return
+    if args.only:
+        run_only(args)
+        return
+    run_ours(args, rank, local_rank, world)
+
+
+if __name__ == "__main__":
+    main()

@@ -22,7 +22,7 @@ US_ENCODE_HOST_ONLY = 1
 US_ENCODE_SORT_ROWS = 2
 
 EXPORTS = ["us_encode", "us_get_stats", "us_decode", "us_get_row_order", "us_spmm",
-           "us_last_error", "us_destroy", "us_spmm_bytes", "us_launch_info", "us_status_string"]
+           "us_last_error", "us_stage_timers", "us_destroy", "us_spmm_bytes", "us_launch_info", "us_status_string"]
 
 
 class us_format(ctypes.Structure):
@@ -46,6 +46,7 @@ _lib.us_get_row_order.argtypes = [_vp, _vp]
 _lib.us_spmm.argtypes = [_vp, _vp, ctypes.c_int32, _vp, _vp, _vp]
 _lib.us_last_error.argtypes = [_vp]
 _lib.us_destroy.argtypes = [_vp]
+_lib.us_stage_timers.argtypes = [_vp, ctypes.c_int32, _vp]
 _lib.us_spmm_bytes.argtypes = [_vp, ctypes.c_int32, ctypes.c_int32]
 _lib.us_spmm_bytes.restype = ctypes.c_int64
 _lib.us_launch_info.argtypes = [_vp, ctypes.c_int32] + [ctypes.POINTER(ctypes.c_int32)] * 3
@@ -115,6 +116,16 @@ def us_spmm(h: int, X_ptr: int, N: int, x_scale_ptr: int | None, Y_ptr: int, str
 
 def us_last_error(h: int) -> int:
     return int(_lib.us_last_error(h))
+
+
+def us_stage_timers(h: int, enable: int = -1, read: bool = False):
+    """Switch the kernel's stage timers on/off; with read=True return (and clear) the sums
+    {wait, decode, epilogue, lifetime} in SM cycles plus the number of warps."""
+    out = (ctypes.c_uint64 * 5)() if read else None
+    _check(_lib.us_stage_timers(h, int(enable), out), "us_stage_timers")
+    if read:
+        return dict(zip(("wait", "decode", "epilogue", "lifetime", "warps"), [int(v) for v in out]))
+    return None
 
 
 def us_destroy(h: int):

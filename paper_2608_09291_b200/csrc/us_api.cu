@@ -23,6 +23,8 @@ struct us_handle {
     int32_t* d_acc = nullptr;
     uint32_t* d_cnt = nullptr;
     uint32_t* d_err = nullptr;
+    unsigned long long* d_timers = nullptr;
+    bool timers_on = false;
     cudaError_t sticky = cudaSuccess;
 };
 
@@ -59,18 +61,36 @@ bool plan_launch(const us_handle* h, int N, LaunchGeom* g)
 template <int NT>
 cudaError_t launch_nt(const us::SpmmParams& p, int grid, int block, int smem, cudaStream_t st)
 {
-    auto kern = us::us_spmm_kernel<NT, kStages>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
-    kern<<<grid, block, smem, st>>>(p);
+    if (p.mask_rows % 2 == 0)
+        us::us_spmm_kernel<NT, kStages, 2><<<grid, block, smem, st>>>(p);
+    else
+        us::us_spmm_kernel<NT, kStages, 1><<<grid, block, smem, st>>>(p);
     return cudaGetLastError();
+}
+
+// Opt every kernel variant in to the device's full dynamic shared memory (once per handle, at
+// encode time, so that us_spmm itself is nothing but a launch).
+template <int NT>
+cudaError_t enable_large_smem_nt(int bytes)
+{
+    cudaError_t e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, kStages, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, kStages, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    return e;
+}
+cudaError_t enable_large_smem(int bytes)
+{
+    cudaError_t e = enable_large_smem_nt<1>(bytes);
+    if (e == cudaSuccess) e = enable_large_smem_nt<2>(bytes);
+    if (e == cudaSuccess) e = enable_large_smem_nt<4>(bytes);
+    if (e == cudaSuccess) e = enable_large_smem_nt<8>(bytes);
+    return e;
 }
 
 void free_device(us_handle* h)
 {
     cudaFree(h->d_blob); cudaFree(h->d_item_off); cudaFree(h->d_cta_begin);
     cudaFree(h->d_row_order); cudaFree(h->d_w_scale); cudaFree(h->d_acc);
-    cudaFree(h->d_cnt); cudaFree(h->d_err);
+    cudaFree(h->d_cnt); cudaFree(h->d_err); cudaFree(h->d_timers);
 }
 
 template <class T>
@@ -107,6 +127,7 @@ us_status us_encode(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_sca
     cudaError_t e = cudaGetDevice(&h->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device);
+    if (e == cudaSuccess) e = enable_large_smem(h->max_smem);
     if (e != cudaSuccess) { delete h; return US_ERR_CUDA; }
 
     const us::HostMatrix& hm = h->host;
@@ -193,6 +214,7 @@ us_status us_spmm(us_handle* h, const void* X, int32_t N, const void* x_scale, v
     p.X = static_cast<const uint8_t*>(X);
     p.x_scale = static_cast<const uint16_t*>(x_scale);
     p.Y = Y; p.acc = h->d_acc; p.cnt = h->d_cnt; p.err = h->d_err;
+    p.timers = h->timers_on ? h->d_timers : nullptr;
     p.M = (int32_t)hm.M; p.K = (int32_t)hm.K; p.N = N;
     p.n_strips = (int32_t)hm.n_strips; p.n_segs = (int32_t)hm.n_segs;
     p.nkb = hm.nkb; p.mask_rows = hm.mask_rows; p.K_L = hm.fmt.K_L;
@@ -224,6 +246,23 @@ us_status us_last_error(us_handle* h)
     if (e != cudaSuccess) return US_ERR_CUDA;
     if (flag == us::kErrTimeout) return US_ERR_DEVICE_TIMEOUT;
     return flag ? US_ERR_CUDA : US_OK;
+}
+
+us_status us_stage_timers(us_handle* h, int32_t enable, uint64_t* out5)
+{
+    if (!h) return US_ERR_INVALID_ARG;
+    if (!h->on_device) return US_ERR_UNSUPPORTED;
+    if (!h->d_timers) {
+        if (cudaMalloc((void**)&h->d_timers, 8 * sizeof(unsigned long long)) != cudaSuccess) return US_ERR_ALLOC;
+        cudaMemset(h->d_timers, 0, 8 * sizeof(unsigned long long));
+    }
+    if (out5) {
+        if (cudaDeviceSynchronize() != cudaSuccess) return US_ERR_CUDA;
+        if (cudaMemcpy(out5, h->d_timers, 5 * sizeof(uint64_t), cudaMemcpyDeviceToHost) != cudaSuccess) return US_ERR_CUDA;
+        cudaMemset(h->d_timers, 0, 8 * sizeof(unsigned long long));
+    }
+    if (enable >= 0) h->timers_on = enable != 0;
+    return US_OK;
 }
 
 us_status us_destroy(us_handle* h)
