@@ -441,7 +441,8 @@ def run_only(args):
     for sw in case.sw:
         for k, v in binding.us_stage_timers(sw.handle, 0, read=True).items():
             tm[k] = tm.get(k, 0) + v
-    timers = {k: (v / tm["warps"] if k != "warps" else v / len(case.sw)) for k, v in tm.items()}
+    per_warp = ("wait", "decode", "epilogue", "lifetime", "prologue")
+    timers = {k: (v / tm["warps"] if k in per_warp else v / len(case.sw)) for k, v in tm.items()}
     print(json.dumps({"only": args.only, "us_per_launch_stream_order": t * 1e6, "alg_bytes": alg,
                       "stored_bytes": binding.us_spmm_bytes(case.sw[0].handle, N, fp16),
                       "gbs": alg / t / 1e9, "replicas": len(case.sw), "format": list(case.stats["fmt"]),

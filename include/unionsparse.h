@@ -123,12 +123,14 @@ us_status us_last_error(us_handle* h);
 /*
  * Diagnostic stage timers of the SpMM kernel (paper Sec. VII-C reports where its kernel's time
  * goes; these are the same question asked of this one). enable: 1 = record in later us_spmm
- * calls, 0 = stop, -1 = leave as is. out5 (host, may be NULL): synchronises the device, returns
- * and clears five sums over all warps that ran since the last read -- SM cycles spent waiting for
- * staged tiles, decoding + MMA, in the reduce/store epilogue, whole warp lifetime, and the number
- * of warps. Recording costs a few clock reads per tile; off by default.
+ * calls, 0 = stop, -1 = leave as is. out8 (host, may be NULL): synchronises the device, returns
+ * and clears eight figures over all warps that ran since the last read -- sums of SM cycles spent
+ * [0] waiting for staged tiles, [1] decoding + MMA, [2] in the reduce/store epilogue, [3] whole
+ * warp lifetime; [4] the number of warps; [5] sum of cycles before a warp's first tile; [6] the
+ * longest warp lifetime in cycles; [7] nanoseconds from the first warp's start to the last
+ * warp's end. Recording costs a few clock reads per tile; off by default.
  */
-us_status us_stage_timers(us_handle* h, int32_t enable, uint64_t* out5);
+us_status us_stage_timers(us_handle* h, int32_t enable, uint64_t* out8);
 
 /* Frees device and host memory. NULL is accepted. */
 us_status us_destroy(us_handle* h);

@@ -120,11 +120,13 @@ def us_last_error(h: int) -> int:
 
 def us_stage_timers(h: int, enable: int = -1, read: bool = False):
     """Switch the kernel's stage timers on/off; with read=True return (and clear) the sums
-    {wait, decode, epilogue, lifetime} in SM cycles plus the number of warps."""
-    out = (ctypes.c_uint64 * 5)() if read else None
+    {wait, decode, epilogue, lifetime, prologue} in SM cycles, the number of warps, the
+    longest warp lifetime and the first-start-to-last-end span in ns."""
+    out = (ctypes.c_uint64 * 8)() if read else None
     _check(_lib.us_stage_timers(h, int(enable), out), "us_stage_timers")
     if read:
-        return dict(zip(("wait", "decode", "epilogue", "lifetime", "warps"), [int(v) for v in out]))
+        return dict(zip(("wait", "decode", "epilogue", "lifetime", "warps", "prologue", "max_lifetime", "span_ns"),
+                        [int(v) for v in out]))
     return None
 
 

@@ -18,6 +18,7 @@ def nvcc_command(out: Path, verbose: bool = False) -> list[str]:
            "-Xcompiler", "-fPIC,-O3,-Wall", "-shared", "-cudart", "shared"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
+    cmd += os.environ.get("US_NVCC_FLAGS", "").split()
     return cmd + [str(s) for s in SOURCES] + ["-o", str(out)]
 
 

@@ -1,6 +1,7 @@
 // C ABI of the library (declared in include/unionsparse.h): handle management, upload, launch.
 #include <algorithm>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -17,7 +18,9 @@ struct us_handle {
     int max_smem = 0;
     uint8_t* d_blob = nullptr;
     uint32_t* d_item_off = nullptr;
-    uint32_t* d_cta_begin = nullptr;
+    std::vector<uint32_t> cta_begin[4];  // schedule per N class (NT = 1, 2, 4, 8)
+    int G[4] = {1, 1, 1, 1};          // segments per K range, per class
+    int s_local[4] = {0, 0, 0, 0};    // strips held in shared memory (0 = direct mode), per class
     int32_t* d_row_order = nullptr;
     uint16_t* d_w_scale = nullptr;
     int32_t* d_acc = nullptr;
@@ -31,50 +34,113 @@ struct us_handle {
 namespace {
 
 constexpr int kStages = 2;
-constexpr int kMaxWarps = 16;
 constexpr int kMinWarps = 2;
 
 int nt_for(int N) { return N <= 8 ? 1 : N <= 16 ? 2 : N <= 32 ? 4 : 8; }
+int class_of(int nt) { return nt == 1 ? 0 : nt == 2 ? 1 : nt == 4 ? 2 : 3; }
+
+// Tuning knobs, overridable from the environment (read once per process) for experiments.
+int env_int(const char* name, int fallback)
+{
+    const char* v = std::getenv(name);
+    return (v && *v) ? std::atoi(v) : fallback;
+}
+int x_budget() { static int v = env_int("US_X_BUDGET_KB", 66) * 1024; return v; }          // int8 X of one K range
+int local_acc_budget() { static int v = env_int("US_LOCAL_ACC_KB", 16) * 1024; return v; }  // local strip sums
+int max_warps() { static int v = std::min(16, std::max(2, env_int("US_MAX_WARPS", 16))); return v; }
 
 struct LaunchGeom {
-    int nt, warps, smem;
+    int nt, cls, warps, smem;
     uint32_t slot_bytes;
 };
 
-// Shared-memory layout of us_spmm_kernel: selector table, int8 X segment, per-token sums,
-// mbarriers, claim counter, then the per-warp rings.
+// Segments per K range for an N class: as many as keep the int8 activations within kXBudget.
+int segs_per_range(const us::HostMatrix& hm, int nt)
+{
+    int g = (x_budget() / (nt * 8) - 32) / hm.fmt.K_L;
+    return (int)std::max<int64_t>(1, std::min<int64_t>(g, hm.n_segs));
+}
+
+// Shared-memory layout of us_spmm_kernel: selector table, int8 X of one K range, per-(segment,
+// token) sums, mbarriers, claim counter, local strip accumulators + counters, per-warp rings.
 bool plan_launch(const us_handle* h, int N, LaunchGeom* g)
 {
     g->nt = nt_for(N);
+    g->cls = class_of(g->nt);
+    const int G = h->G[g->cls], s_local = h->s_local[g->cls];
     g->slot_bytes = (h->host.max_item_bytes + 256u + 127u) & ~127u;
-    const int fixed = (int)us::kLutBytes + g->nt * 8 * (h->host.fmt.K_L + 32) + 64 * 4 +
-                      32 * kStages * 8 + 32 * 4 + 128;
+    const int fixed = (int)us::kLutBytes + g->nt * 8 * (G * h->host.fmt.K_L + 32) + G * g->nt * 8 * 4 +
+                      32 * kStages * 8 + 32 * 4 + s_local * (g->nt * 128 + 1) * 4 + 2 * us::kOffTable * 4 + 128;
     const int limit = h->max_smem > 0 ? h->max_smem : 227 * 1024;
     int warps = (limit - fixed) / (int)(kStages * g->slot_bytes);
-    warps = std::min(warps, kMaxWarps);
+    warps = std::min(warps, max_warps());
     if (warps < kMinWarps) return false;
     g->warps = warps;
     g->smem = fixed + warps * kStages * (int)g->slot_bytes;
     return true;
 }
 
+// Chooses, per N class, the K-range width and whether strips are summed in shared memory.
+void plan_classes(us_handle* h, int n_cta, std::vector<uint32_t> (&sched)[4])
+{
+    for (int c = 0; c < 4; ++c) {
+        const int nt = 1 << c;
+        int G = segs_per_range(h->host, nt), worst = 1;
+        us::make_schedule(h->host, n_cta, G, &sched[c], &worst);
+        if (G > 1 && worst * nt * 512 <= local_acc_budget()) {
+            h->G[c] = G;
+            h->s_local[c] = worst;
+        } else {  // direct mode: one segment per range, every tile goes to the global workspace
+            h->G[c] = 1;
+            h->s_local[c] = 0;
+            if (G != 1) us::make_schedule(h->host, n_cta, 1, &sched[c], &worst);
+        }
+    }
+}
+
+int chains_knob() { static int v = env_int("US_CHAINS", 1); return v; }
+int run_knob() { static int v = env_int("US_RUN", 0); return v; }
+
+// decode chains per tile: as many as the knob asks for and the tile's mask words divide into
+int chains_for(int mask_rows)
+{
+    const int want = chains_knob();
+    if (want >= 2 && mask_rows % 2 == 0) return 2;
+    return 1;
+}
+
+template <int NT, int CH>
+cudaError_t launch_ch(const us::SpmmParams& p, int grid, int block, int smem, cudaStream_t st)
+{
+    if (p.s_local > 0) us::us_spmm_kernel<NT, kStages, CH, true><<<grid, block, smem, st>>>(p);
+    else us::us_spmm_kernel<NT, kStages, CH, false><<<grid, block, smem, st>>>(p);
+    return cudaGetLastError();
+}
+
 template <int NT>
 cudaError_t launch_nt(const us::SpmmParams& p, int grid, int block, int smem, cudaStream_t st)
 {
-    if (p.mask_rows % 2 == 0)
-        us::us_spmm_kernel<NT, kStages, 2><<<grid, block, smem, st>>>(p);
-    else
-        us::us_spmm_kernel<NT, kStages, 1><<<grid, block, smem, st>>>(p);
-    return cudaGetLastError();
+    switch (chains_for(p.mask_rows)) {
+        case 2: return launch_ch<NT, 2>(p, grid, block, smem, st);
+        default: return launch_ch<NT, 1>(p, grid, block, smem, st);
+    }
 }
 
 // Opt every kernel variant in to the device's full dynamic shared memory (once per handle, at
 // encode time, so that us_spmm itself is nothing but a launch).
+template <int NT, int CH>
+cudaError_t enable_large_smem_ch(int bytes)
+{
+    const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
+    cudaError_t e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, kStages, CH, true>, attr, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, kStages, CH, false>, attr, bytes);
+    return e;
+}
 template <int NT>
 cudaError_t enable_large_smem_nt(int bytes)
 {
-    cudaError_t e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, kStages, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, kStages, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    cudaError_t e = enable_large_smem_ch<NT, 1>(bytes);
+    if (e == cudaSuccess) e = enable_large_smem_ch<NT, 2>(bytes);
     return e;
 }
 cudaError_t enable_large_smem(int bytes)
@@ -88,7 +154,7 @@ cudaError_t enable_large_smem(int bytes)
 
 void free_device(us_handle* h)
 {
-    cudaFree(h->d_blob); cudaFree(h->d_item_off); cudaFree(h->d_cta_begin);
+    cudaFree(h->d_blob); cudaFree(h->d_item_off);
     cudaFree(h->d_row_order); cudaFree(h->d_w_scale); cudaFree(h->d_acc);
     cudaFree(h->d_cnt); cudaFree(h->d_err); cudaFree(h->d_timers);
 }
@@ -122,23 +188,33 @@ us_status us_encode(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_sca
         s = US_ERR_ALLOC;
     }
     if (s != US_OK) { delete h; return s; }
-    if (flags & US_ENCODE_HOST_ONLY) { *out = h; return US_OK; }
+    if (h->host.n_items >= (1 << 24) || h->host.n_strips * h->host.n_segs >= (1 << 24) || h->host.n_segs >= (1 << 16)) {
+        delete h;
+        return US_ERR_UNSUPPORTED;  // the kernel's index arithmetic assumes fewer tiles
+    }
+    if (flags & US_ENCODE_HOST_ONLY) {
+        std::vector<uint32_t> sched[4];
+        plan_classes(h, 148, sched);
+        *out = h;
+        return US_OK;
+    }
 
     cudaError_t e = cudaGetDevice(&h->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device);
+    if (e == cudaSuccess && h->sm_count > us::kMaxCtas) h->sm_count = us::kMaxCtas;
     if (e == cudaSuccess) e = enable_large_smem(h->max_smem);
     if (e != cudaSuccess) { delete h; return US_ERR_CUDA; }
 
     const us::HostMatrix& hm = h->host;
-    std::vector<uint32_t> sched;
-    us::make_schedule(hm, h->sm_count, &sched);
+    std::vector<uint32_t> sched[4];
+    plan_classes(h, h->sm_count, sched);
     const int nt_max = nt_for(max_N);
     const size_t acc_bytes = (size_t)hm.n_strips * nt_max * 128 * sizeof(int32_t);
     const size_t cnt_bytes = (size_t)hm.n_strips * sizeof(uint32_t);
     e = upload(&h->d_blob, hm.blob.data(), hm.blob.size());
     if (e == cudaSuccess) e = upload(&h->d_item_off, hm.item_off.data(), hm.item_off.size() * 4);
-    if (e == cudaSuccess) e = upload(&h->d_cta_begin, sched.data(), sched.size() * 4);
+    for (int c = 0; c < 4; ++c) h->cta_begin[c] = sched[c];
     if (e == cudaSuccess) e = upload(&h->d_row_order, hm.row_order.data(), hm.row_order.size() * 4);
     if (e == cudaSuccess && !hm.w_scale.empty()) e = upload(&h->d_w_scale, hm.w_scale.data(), hm.w_scale.size() * 2);
     if (e == cudaSuccess) e = cudaMalloc((void**)&h->d_acc, acc_bytes);
@@ -209,7 +285,21 @@ us_status us_spmm(us_handle* h, const void* X, int32_t N, const void* x_scale, v
 
     const us::HostMatrix& hm = h->host;
     us::SpmmParams p;
-    p.blob = h->d_blob; p.item_off = h->d_item_off; p.cta_begin = h->d_cta_begin;
+    p.blob = h->d_blob; p.item_off = h->d_item_off;
+    std::memcpy(p.cta_begin, h->cta_begin[g.cls].data(), h->cta_begin[g.cls].size() * sizeof(uint32_t));
+    p.G = h->G[g.cls]; p.s_local = h->s_local[g.cls];
+    {
+        const int64_t n_kr = (hm.n_segs + p.G - 1) / p.G;
+        const int64_t g_last = hm.n_segs - (n_kr - 1) * p.G;
+        auto magic = [](uint64_t d) { return ((1ull << 40) / d) + 1ull; };
+        p.mg_g = magic((uint64_t)p.G);
+        p.mg_glast = magic((uint64_t)g_last);
+        p.mg_krs = magic((uint64_t)hm.n_strips * (uint64_t)p.G);
+        // claim runs of up to half a strip's segments of the range, so that a CTA's warps still
+        // share its strips evenly
+        const int want = run_knob() > 0 ? run_knob() : std::max(1, p.G / 2);
+        p.run_len = std::max(1, std::min(want, p.G));
+    }
     p.row_order = h->d_row_order; p.w_scale = h->d_w_scale;
     p.X = static_cast<const uint8_t*>(X);
     p.x_scale = static_cast<const uint16_t*>(x_scale);
@@ -219,7 +309,7 @@ us_status us_spmm(us_handle* h, const void* X, int32_t N, const void* x_scale, v
     p.n_strips = (int32_t)hm.n_strips; p.n_segs = (int32_t)hm.n_segs;
     p.nkb = hm.nkb; p.mask_rows = hm.mask_rows; p.K_L = hm.fmt.K_L;
     p.slot_bytes = g.slot_bytes;
-    p.x_fast = (hm.K % 8 == 0) ? 1 : 0;
+    p.x_fast = (hm.K % 32 == 0) ? 2 : (hm.K % 8 == 0) ? 1 : 0;
     p.fp16_out = x_scale ? 1 : 0;
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -248,18 +338,42 @@ us_status us_last_error(us_handle* h)
     return flag ? US_ERR_CUDA : US_OK;
 }
 
-us_status us_stage_timers(us_handle* h, int32_t enable, uint64_t* out5)
+static cudaError_t reset_timers(unsigned long long* d)
+{
+    static unsigned long long z[16 + 4 * us::kMaxCtas];
+    std::memset(z, 0, sizeof(z));
+    z[7] = ~0ull;  // running minimum of the start time stamps
+    return cudaMemcpy(d, z, sizeof(z), cudaMemcpyHostToDevice);
+}
+
+us_status us_stage_timers(us_handle* h, int32_t enable, uint64_t* out8)
 {
     if (!h) return US_ERR_INVALID_ARG;
     if (!h->on_device) return US_ERR_UNSUPPORTED;
     if (!h->d_timers) {
-        if (cudaMalloc((void**)&h->d_timers, 8 * sizeof(unsigned long long)) != cudaSuccess) return US_ERR_ALLOC;
-        cudaMemset(h->d_timers, 0, 8 * sizeof(unsigned long long));
+        if (cudaMalloc((void**)&h->d_timers, (16 + 4 * us::kMaxCtas) * sizeof(unsigned long long)) != cudaSuccess) return US_ERR_ALLOC;
+        reset_timers(h->d_timers);
     }
-    if (out5) {
+    if (out8) {
         if (cudaDeviceSynchronize() != cudaSuccess) return US_ERR_CUDA;
-        if (cudaMemcpy(out5, h->d_timers, 5 * sizeof(uint64_t), cudaMemcpyDeviceToHost) != cudaSuccess) return US_ERR_CUDA;
-        cudaMemset(h->d_timers, 0, 8 * sizeof(unsigned long long));
+        static uint64_t t[16 + 4 * us::kMaxCtas];
+        if (cudaMemcpy(t, h->d_timers, sizeof(t), cudaMemcpyDeviceToHost) != cudaSuccess) return US_ERR_CUDA;
+        if (const char* path = std::getenv("US_TIMER_DUMP")) {
+            if (FILE* f = std::fopen(path, "a")) {
+                for (int c = 0; c < us::kMaxCtas; ++c)
+                    if (t[16 + 4 * c])
+                        std::fprintf(f, "%d %llu %llu %llu %lld\n", c, (unsigned long long)t[16 + 4 * c], (unsigned long long)t[17 + 4 * c],
+                                     (unsigned long long)t[18 + 4 * c], (long long)(t[19 + 4 * c] - t[7]));
+                std::fprintf(f, "#\n");
+                std::fclose(f);
+            }
+        }
+        for (int i = 0; i < 7; ++i) out8[i] = t[i];
+        out8[7] = t[8] > t[7] ? t[8] - t[7] : 0;   // first warp start to last warp end, ns
+        if (std::getenv("US_TIMER_DEBUG") && t[4])
+            std::fprintf(stderr, "[us] prologue checkpoints (cycles/warp): range known %.0f, copies issued %.0f, table done %.0f, X staged %.0f\n",
+                         (double)t[9] / t[4], (double)t[10] / t[4], (double)t[11] / t[4], (double)t[12] / t[4]);
+        reset_timers(h->d_timers);
     }
     if (enable >= 0) h->timers_on = enable != 0;
     return US_OK;

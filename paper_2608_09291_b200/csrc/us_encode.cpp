@@ -135,7 +135,7 @@ us_status encode_host(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_s
             int maxlen = 0;
             for (int l = 0; l < 32; ++l) { maxlen = std::max(maxlen, len[l]); my_P += len[l]; }
             const int J = (maxlen + 3) / 4;
-            std::vector<uint8_t>& b = blobs[sg * h.n_strips + rb];
+            std::vector<uint8_t>& b = blobs[rb * h.n_segs + sg];
             b.assign((size_t)mask_bytes + (size_t)J * 128, 0);
             for (int l = 0; l < 32; ++l) {
                 for (int w = 0; w < mask_rows; ++w)
@@ -181,7 +181,7 @@ void decode_host(const HostMatrix& h, int8_t* W_out)
     std::memset(W_out, 0, (size_t)(h.M * h.K));
     const int nkb = h.nkb, mask_rows = h.mask_rows, K_L = h.fmt.K_L;
     for (int64_t t = 0; t < h.n_items; ++t) {
-        const int64_t sg = t / h.n_strips, rb = t % h.n_strips;
+        const int64_t rb = t / h.n_segs, sg = t % h.n_segs;
         const uint8_t* b = h.blob.data() + (size_t)h.item_off[t] * 16;
         const uint8_t* pay = b + (size_t)mask_rows * 128;
         for (int lane = 0; lane < 32; ++lane) {
@@ -223,17 +223,45 @@ void fill_stats(const HostMatrix& h, us_stats* st)
     st->fmt = h.fmt;
 }
 
-void make_schedule(const HostMatrix& h, int n_cta, std::vector<uint32_t>* begin)
+void make_schedule(const HostMatrix& h, int n_cta, int G, std::vector<uint32_t>* begin,
+                   int* max_local_strips)
 {
+    // Processing order: K range kr (G segments, the last one possibly shorter), then strip, then
+    // segment within the range. Position u of that order maps to tile rb * n_segs + kr * G + sgl.
     begin->assign((size_t)n_cta + 1, 0);
-    const uint64_t total = h.item_off[h.n_items];
-    int64_t t = 0;
+    const int64_t n_kr = (h.n_segs + G - 1) / G;
+    std::vector<uint64_t> prefix((size_t)h.n_items + 1, 0);
+    std::vector<int32_t> strip_of((size_t)h.n_items), kr_of((size_t)h.n_items);
+    int64_t u = 0;
+    for (int64_t kr = 0; kr < n_kr; ++kr) {
+        const int64_t g_kr = std::min<int64_t>(G, h.n_segs - kr * G);
+        for (int64_t rb = 0; rb < h.n_strips; ++rb)
+            for (int64_t sgl = 0; sgl < g_kr; ++sgl, ++u) {
+                const int64_t t = rb * h.n_segs + kr * G + sgl;
+                prefix[u + 1] = prefix[u] + (h.item_off[t + 1] - h.item_off[t]);
+                strip_of[u] = (int32_t)rb;
+                kr_of[u] = (int32_t)kr;
+            }
+    }
+    const uint64_t total = prefix[h.n_items];
+    int64_t pos = 0;
     for (int c = 0; c <= n_cta; ++c) {
         const uint64_t target = total * (uint64_t)c / (uint64_t)n_cta;
-        while (t < h.n_items && h.item_off[t] < target) ++t;
-        (*begin)[c] = (uint32_t)t;
+        while (pos < h.n_items && prefix[pos] < target) ++pos;
+        (*begin)[c] = (uint32_t)pos;
     }
     (*begin)[n_cta] = (uint32_t)h.n_items;
+    int worst = 1;
+    for (int c = 0; c < n_cta; ++c) {
+        int64_t a = (*begin)[c], b = (*begin)[c + 1];
+        while (a < b) {  // one K range at a time
+            int64_t e = a;
+            while (e < b && kr_of[e] == kr_of[a]) ++e;
+            worst = std::max(worst, strip_of[e - 1] - strip_of[a] + 1);
+            a = e;
+        }
+    }
+    if (max_local_strips) *max_local_strips = worst;
 }
 
 }  // namespace us

@@ -3,7 +3,7 @@
 // Layout ("lane-stream" IE-BME, H_L = 16, R_A = 2, C_A = 1, paper Sec. V-A with the in-tile
 // order chosen for the sm_100a kernel):
 //   * rows are cut into strips of 16 (after an optional row order); columns into segments of
-//     K_L; one (segment, strip) pair is a tile ("item"), tiles ordered segment-major.
+//     K_L; one (strip, segment) pair is a tile ("item"), tile index = strip * n_segs + segment.
 //   * a tile is decoded by one warp; lane l = 4*g + t owns, for every 32-column k-block kb of
 //     the tile, the 8 columns 32*kb + 8*t + j (j = 0..7) of strip rows g and g+8 -- exactly
 //     the A-fragment slots of that lane in an m16n8k32 integer MMA.
@@ -44,9 +44,11 @@ us_status encode_host(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_s
 void decode_host(const HostMatrix& h, int8_t* W_out);
 void fill_stats(const HostMatrix& h, us_stats* st);
 
-// Byte-balanced split of the tile sequence over `n_cta` persistent CTAs: CTA c processes tiles
-// [begin[c], begin[c+1]). `begin` has n_cta + 1 entries.
-void make_schedule(const HostMatrix& h, int n_cta, std::vector<uint32_t>* begin);
+// Byte-balanced split of the processing order (K range of G segments, strip, segment) over
+// `n_cta` persistent CTAs: CTA c processes positions [begin[c], begin[c+1]) (n_cta + 1 entries).
+// max_local_strips = the most strips any CTA touches within one K range.
+void make_schedule(const HostMatrix& h, int n_cta, int G, std::vector<uint32_t>* begin,
+                   int* max_local_strips);
 
 // Default K_L for a shape when the caller passes no format.
 int32_t default_K_L(int64_t M, int64_t K);

@@ -1,13 +1,15 @@
 // sm_100a SpMM kernel: lane-stream IE-BME weights (see us_host.h) x dense INT4 activations.
 //
 // Steps of the hot path (paper Alg. 2 / Sec. VI, re-designed for B200):
-//   schedule   persistent CTAs, one per SM; CTA c owns tiles [cta_begin[c], cta_begin[c+1]) of
-//              the segment-major tile sequence (byte balanced on the host); warps claim tiles
-//              from a shared-memory counter.
+//   schedule   persistent CTAs, one per SM. The K segments are grouped into K ranges of G
+//              segments whose activations fit in shared memory; tiles are processed in the
+//              order (K range, strip, segment) and CTA c owns positions [cta_begin[c],
+//              cta_begin[c+1]) of that sequence (byte balanced on the host). Warps claim
+//              tiles from a shared-memory counter, one tile ahead of the copy they issue.
 //   stage W    every warp runs its own ring of STAGES slots; one cp.async.bulk per tile
 //              (bitmaps + payload are one contiguous blob) completing on an mbarrier
 //              (the role of the paper's double-buffered producer/consumer pipeline, Sec. VI-A).
-//   stage X    the CTA expands the INT4 activations of the current K segment once into int8
+//   stage X    the CTA expands the INT4 activations of the current K range once into int8
 //              (x16, so no per-element sign extension) in shared memory.
 //   decode     bitmap -> operand fragment (the role of LSPD, Sec. VI-B): per lane and k-block
 //              one mask byte indexes a 256-entry selector table; two byte-permutes deposit the
@@ -16,20 +18,27 @@
 //   MMA        mma.sync m16n8k32 s8: fragment rows g carry the raw payload bytes
 //              (16*w_hi + (w_lo+8)), rows g+8 the low nibbles (w_lo+8); with Sx = sum_k x,
 //              Y_lo = E - 8*Sx and Y_hi = (RAW - E)/16, all exact in INT32.
-//   reduce     split-K partial sums go to an INT32 workspace with red.add; the warp whose
-//              arrival completes a strip reads the sums, applies the optional fp16 dequant
-//              epilogue, stores Y and leaves workspace and counter zeroed.
+//   reduce     (local mode) tiles of one strip are summed in a shared-memory accumulator; the
+//              warp that adds the CTA's last tile of a strip flushes it: straight to Y when the
+//              CTA saw every segment of the strip, else into the global INT32 workspace.
+//              (direct mode, used when a CTA would touch too many strips) every tile goes to
+//              the global workspace with red.add. In both, the arrival that completes a strip
+//              reads the sums, applies the optional fp16 dequant epilogue, stores Y and leaves
+//              workspace and counter zeroed.
 #pragma once
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <type_traits>
+
 namespace us {
+
+constexpr int kMaxCtas = 192;   // persistent CTAs (one per SM) the schedule can describe
 
 struct SpmmParams {
     const uint8_t* blob;
     const uint32_t* item_off;   // n_items + 1, units of 16 bytes
-    const uint32_t* cta_begin;  // gridDim.x + 1
     const int32_t* row_order;   // Mp entries
     const uint16_t* w_scale;    // M fp16 bit patterns or nullptr
     const uint8_t* X;           // N x ceil(K/2) packed INT4
@@ -38,51 +47,53 @@ struct SpmmParams {
     int32_t* acc;               // split-K workspace, zero between calls
     uint32_t* cnt;              // per-strip arrival counters, zero between calls
     uint32_t* err;              // device error word
-    unsigned long long* timers; // optional stage timers (5 counters) or nullptr
+    unsigned long long* timers; // optional stage timers (9 counters) or nullptr
     int32_t M, K, N;
     int32_t n_strips, n_segs;
+    int32_t G;                  // segments per K range
+    int32_t run_len;            // consecutive positions a warp claims at a time
+    unsigned long long mg_g, mg_glast, mg_krs;  // floor(2^40/d)+1 for d = G, the last range's
+                                                // segment count, n_strips * G
+    int32_t s_local;            // local mode: strips a CTA may hold in shared memory (0 = direct mode)
     int32_t nkb, mask_rows, K_L;
     uint32_t slot_bytes;        // ring slot size (max tile blob + slack), multiple of 128
-    int32_t x_fast;             // X rows are 4-byte aligned and K % 8 == 0
+    int32_t x_fast;             // 2: K % 32 == 0 (16-byte loads); 1: K % 8 == 0 (4-byte loads); 0: bytes
     int32_t fp16_out;
+    // CTA c owns positions [cta_begin[c], cta_begin[c+1]) of the (K range, strip, segment) order.
+    // Kept in the kernel parameters: the schedule is known without a global-memory round trip.
+    uint32_t cta_begin[kMaxCtas + 1];
 };
 
 constexpr uint32_t kLutBytes = 256 * 32 * 4;
 constexpr uint32_t kFill = 0x08080808u;
 constexpr uint32_t kErrTimeout = 1;
+constexpr int kNoRow = -2;        // "row ids not loaded yet" marker (-1 is a padding row)
+constexpr int kOffTable = 384;   // tile offsets of a CTA kept in shared memory (start, end pairs)
 
 // ---- selector table -------------------------------------------------------------------------
 // entry(m): low 16 bits  = prmt selector for mask bits 0..3 reading the 4 bytes AT the lane's
 //                          stream position (nibble j = rank of bit j, or 4 = neutral byte);
 //           high 16 bits = prmt selector for mask bits 4..7 reading the 4 bytes that END at the
 //                          stream position after this k-block (nibble j = 4 - c_hi + rank).
-struct LutTable {
-    uint32_t v[256];
-};
-constexpr LutTable make_lut()
+__host__ __device__ constexpr uint32_t lut_entry(int m)
 {
-    LutTable t{};
-    for (int m = 0; m < 256; ++m) {
-        uint32_t lo = 0, hi = 0;
-        int rank = 0;
-        for (int j = 0; j < 4; ++j) {
-            uint32_t s = 4;
-            if ((m >> j) & 1) s = rank++;
-            lo |= s << (4 * j);
-        }
-        int c_hi = 0;
-        for (int j = 4; j < 8; ++j) c_hi += (m >> j) & 1;
-        rank = 0;
-        for (int j = 4; j < 8; ++j) {
-            uint32_t s = 4;
-            if ((m >> j) & 1) s = 4 - c_hi + rank++;
-            hi |= s << (4 * (j - 4));
-        }
-        t.v[m] = lo | (hi << 16);
+    uint32_t lo = 0, hi = 0;
+    int rank = 0;
+    for (int j = 0; j < 4; ++j) {
+        uint32_t s = 4;
+        if ((m >> j) & 1) s = rank++;
+        lo |= s << (4 * j);
     }
-    return t;
+    int c_hi = 0;
+    for (int j = 4; j < 8; ++j) c_hi += (m >> j) & 1;
+    rank = 0;
+    for (int j = 4; j < 8; ++j) {
+        uint32_t s = 4;
+        if ((m >> j) & 1) s = 4 - c_hi + rank++;
+        hi |= s << (4 * (j - 4));
+    }
+    return lo | (hi << 16);
 }
-__constant__ LutTable c_lut = make_lut();
 
 // ---- PTX helpers ----------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p)
@@ -150,45 +161,103 @@ __device__ __forceinline__ void mma_s8(int (&c)[4], uint32_t a0, uint32_t a1, ui
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// ---- X staging: INT4 -> int8 (x16) for one K segment, plus 16 * sum_k x per token -------------
-template <int NT>
-__device__ __forceinline__ void stage_x(const SpmmParams& p, int sg, uint8_t* x8, int32_t* sx16,
-                                        int warp, int lane, int n_warps)
+// ---- shared-memory access by 32-bit address ---------------------------------------------------
+__device__ __forceinline__ uint32_t lds32(uint32_t a)
 {
-    const int xstride = p.K_L + 32;
-    const int words = p.K_L / 8;  // one word = 8 activations
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t a)
+{
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a));
+    return v;
+}
+
+// ---- X staging: INT4 -> int8 (x16) for one K range, plus 16 * sum_k x per (segment, token) -----
+// expands 8 packed activations (one 32-bit word) into two words of int8 (x16) and adds 16 * their sum
+__device__ __forceinline__ uint2 expand8(uint32_t v, int32_t& s)
+{
+    const uint32_t te = (v << 4) & 0xF0F0F0F0u;  // 16*x for k even
+    const uint32_t to = v & 0xF0F0F0F0u;         // 16*x for k odd
+    s = __dp4a((int)te, 0x01010101, s);
+    s = __dp4a((int)to, 0x01010101, s);
+    return make_uint2(prmt(te, to, 0x5140), prmt(te, to, 0x7362));
+}
+
+// sx16 must be zero on entry (the caller clears it and synchronises).
+// Units below `first_unit` (of the 16-byte path) were already staged by the caller.
+template <int NT>
+__device__ __forceinline__ void stage_x(const SpmmParams& p, int seg0, int n_seg, uint8_t* x8,
+                                        int xstride, int32_t* sx16, int first_unit)
+{
     const int64_t ldx = ((int64_t)p.K + 1) / 2;
-    const int64_t k0 = (int64_t)sg * p.K_L;
-    for (int n = warp; n < NT * 8; n += n_warps) {
-        int32_t s = 0;
-        for (int wi = lane; wi < words; wi += 32) {
-            const int64_t k = k0 + 8 * wi;
-            uint32_t v = 0;
-            if (n < p.N) {
-                const uint8_t* src = p.X + (int64_t)n * ldx + k / 2;
-                if (p.x_fast && k + 8 <= p.K) {
-                    v = *reinterpret_cast<const uint32_t*>(src);
-                } else {
-                    for (int e = 0; e < 8; ++e) {
-                        if (k + e < p.K) {
-                            uint32_t byte = src[e >> 1];
-                            v |= ((e & 1) ? (byte >> 4) : (byte & 0xF)) << (4 * e);
-                        }
+    const int rows = NT * 8;
+    if (p.x_fast == 2) {
+        // 16-byte units (32 activations); all loads of a batch are issued before any is used
+        const int upr = p.K_L / 32;                 // units per (segment, token)
+        const int total = rows * n_seg * upr;
+        constexpr int kBatch = 4;
+        for (int u0 = first_unit + threadIdx.x; u0 < total; u0 += kBatch * blockDim.x) {
+            uint4 v[kBatch];
+#pragma unroll
+            for (int b = 0; b < kBatch; ++b) {
+                const int u = u0 + b * blockDim.x;
+                v[b] = make_uint4(0, 0, 0, 0);
+                if (u < total) {
+                    const int pi = u / upr, q = u - pi * upr;
+                    const int sgl = pi / rows, n = pi - sgl * rows;
+                    const int64_t k = (int64_t)(seg0 + sgl) * p.K_L + 32 * q;
+                    if (n < p.N && k < p.K)
+                        v[b] = __ldg(reinterpret_cast<const uint4*>(p.X + (int64_t)n * ldx + k / 2));
+                }
+            }
+#pragma unroll
+            for (int b = 0; b < kBatch; ++b) {
+                const int u = u0 + b * blockDim.x;
+                if (u < total) {
+                    const int pi = u / upr, q = u - pi * upr;
+                    const int sgl = pi / rows, n = pi - sgl * rows;
+                    int32_t s = 0;
+                    uint4 lo, hi;
+                    uint2 t;
+                    t = expand8(v[b].x, s); lo.x = t.x; lo.y = t.y;
+                    t = expand8(v[b].y, s); lo.z = t.x; lo.w = t.y;
+                    t = expand8(v[b].z, s); hi.x = t.x; hi.y = t.y;
+                    t = expand8(v[b].w, s); hi.z = t.x; hi.w = t.y;
+                    uint4* dst = reinterpret_cast<uint4*>(x8 + n * xstride + sgl * p.K_L + 32 * q);
+                    dst[0] = lo; dst[1] = hi;
+                    if (s) atomicAdd(sx16 + pi, s);
+                }
+            }
+        }
+        return;
+    }
+    // general path: 8 activations at a time, any K and alignment
+    const int wpr = p.K_L / 8;
+    const int total = rows * n_seg * wpr;
+    for (int u = threadIdx.x; u < total; u += blockDim.x) {
+        const int pi = u / wpr, wi = u - pi * wpr;
+        const int sgl = pi / rows, n = pi - sgl * rows;
+        const int64_t k = (int64_t)(seg0 + sgl) * p.K_L + 8 * wi;
+        uint32_t v = 0;
+        if (n < p.N) {
+            const uint8_t* src = p.X + (int64_t)n * ldx + k / 2;
+            if (p.x_fast == 1 && k + 8 <= p.K) {
+                v = __ldg(reinterpret_cast<const uint32_t*>(src));
+            } else {
+                for (int e = 0; e < 8; ++e) {
+                    if (k + e < p.K) {
+                        uint32_t byte = src[e >> 1];
+                        v |= ((e & 1) ? (byte >> 4) : (byte & 0xF)) << (4 * e);
                     }
                 }
             }
-            const uint32_t te = (v << 4) & 0xF0F0F0F0u;  // 16*x for k even
-            const uint32_t to = v & 0xF0F0F0F0u;         // 16*x for k odd
-            uint2 o;
-            o.x = prmt(te, to, 0x5140);
-            o.y = prmt(te, to, 0x7362);
-            *reinterpret_cast<uint2*>(x8 + n * xstride + 8 * wi) = o;
-            s = __dp4a((int)te, 0x01010101, s);
-            s = __dp4a((int)to, 0x01010101, s);
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-        if (lane == 0) sx16[n] = s;
+        int32_t s = 0;
+        *reinterpret_cast<uint2*>(x8 + n * xstride + sgl * p.K_L + 8 * wi) = expand8(v, s);
+        if (s) atomicAdd(sx16 + pi, s);
     }
 }
 
@@ -196,91 +265,199 @@ __device__ __forceinline__ void stage_x(const SpmmParams& p, int sg, uint8_t* x8
 // CH independent decode chains walk consecutive ranges of the tile's k-blocks (chain ch starts at
 // the lane-stream position given by the popcount of the mask words before its range); the chains
 // only share the accumulators, so their shared-memory and permute latencies overlap.
+// All addresses are 32-bit shared-memory addresses: slot_a = the staged tile, lut_a = selector
+// table + 4*lane, xb_a = this lane's first B-fragment of the tile's segment.
 template <int NT, int CH>
-__device__ __forceinline__ void process_tile(const uint32_t* __restrict__ slot,
-                                             const uint32_t* __restrict__ lut,
-                                             const uint8_t* __restrict__ x8, int xstride,
-                                             int mask_rows, int lane, int (&c)[NT][4])
+__device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, uint32_t xb_a,
+                                             int xstride, int mask_rows, int lane, int (&c)[NT][4])
 {
-    const int g = lane >> 2, t = lane & 3;
     const int rows_per = mask_rows / CH;
-    const uint32_t* maskp = slot + lane;
-    const uint32_t* payp = slot + mask_rows * 32 + lane;
-    const uint32_t* lutp = lut + lane;
-    const uint8_t* xb = x8 + g * xstride + 8 * t;
+    const uint32_t mask_a = slot_a + 4u * lane;
+    const uint32_t pay_a = slot_a + 128u * mask_rows + 4u * lane;
     uint32_t b8[CH];   // 8 * (byte position in the lane's payload stream), per chain
     uint32_t d0[CH], sel_hi[CH];
     b8[0] = 0;
 #pragma unroll
     for (int ch = 1; ch < CH; ++ch) {
         uint32_t n = 0;
-        for (int w = 0; w < rows_per; ++w) n += (uint32_t)__popc(maskp[((ch - 1) * rows_per + w) * 32]);
+        for (int w = 0; w < rows_per; ++w) n += (uint32_t)__popc(lds32(mask_a + 128u * ((ch - 1) * rows_per + w)));
         b8[ch] = b8[ch - 1] + 8u * n;
     }
 #pragma unroll
     for (int ch = 0; ch < CH; ++ch) d0[ch] = sel_hi[ch] = 0;
 
-    auto finish_block = [&](int ch, int kb, uint32_t prev) {
+    // finish k-block: second permute (mask bits 4..7), low-nibble rows, MMA against its X fragment
+    auto finish_block = [&](int ch, uint32_t xk_a, uint32_t prev, const uint2* xpre) {
         const uint32_t d1 = prmt(prev, kFill, sel_hi[ch]);
         const uint32_t e0 = d0[ch] & 0x0F0F0F0Fu, e1 = d1 & 0x0F0F0F0Fu;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-            const uint2 b = *reinterpret_cast<const uint2*>(xb + nt * 8 * xstride + kb * 32);
+            const uint2 b = xpre ? xpre[nt] : lds64(xk_a + nt * 8 * xstride);
             mma_s8(c[nt], d0[ch], e0, d1, e1, b.x, b.y);
         }
     };
-
-    for (int w = 0; w < rows_per; ++w) {
-        uint32_t mw[CH];
+    constexpr bool kPreX = NT <= 2;   // small N: fetch the X fragments together with the windows
+    // One mask word = four k-blocks per chain. The stream positions of all four follow from the
+    // mask word alone, so every shared-memory load of the word is issued before any is used.
+    auto word = [&](auto first, int w) {
+        constexpr bool kFirst = decltype(first)::value;
+        uint32_t pos[CH][5], wm1[CH][4], w0[CH][4], w1[CH][4], e[CH][4];
+        uint2 xf[CH][4][kPreX ? NT : 1];
 #pragma unroll
-        for (int ch = 0; ch < CH; ++ch) mw[ch] = maskp[(ch * rows_per + w) * 32];
+        for (int ch = 0; ch < CH; ++ch) {
+            const uint32_t mw = lds32(mask_a + 128u * (ch * rows_per + w));
+            pos[ch][0] = b8[ch];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t cum = (i == 3) ? mw : (mw & ((1u << (8 * i + 8)) - 1u));
+                pos[ch][i + 1] = b8[ch] + 8u * (uint32_t)__popc(cum);
+                e[ch][i] = lut_a + prmt(mw, 0u, 0x4440u + i) * 128u;   // address of the table entry
+            }
+            b8[ch] = pos[ch][4];
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
 #pragma unroll
             for (int ch = 0; ch < CH; ++ch) {
-                const uint32_t* q = payp + ((b8[ch] >> 5) << 5);
-                const uint32_t wm1 = *(q - 32), w0 = q[0], w1 = q[32];
-                const uint32_t prev = __funnelshift_r(wm1, w0, b8[ch]);
-                const uint32_t lo = __funnelshift_r(w0, w1, b8[ch]);
-                if (w > 0 || i > 0) finish_block(ch, 4 * (ch * rows_per + w) + i - 1, prev);
-                const uint32_t mb = (mw[ch] >> (8 * i)) & 0xFFu;
-                const uint32_t e = lutp[mb * 32];
-                d0[ch] = prmt(lo, kFill, e);
-                sel_hi[ch] = e >> 16;
-                b8[ch] += 8u * (uint32_t)__popc(mb);
+                const uint32_t a = pay_a + ((pos[ch][i] >> 5) << 7);
+                wm1[ch][i] = lds32(a - 128u);
+                w0[ch][i] = lds32(a);
+                w1[ch][i] = lds32(a + 128u);
+                e[ch][i] = lds32(e[ch][i]);
+                if (kPreX && !(kFirst && i == 0)) {
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt)
+                        xf[ch][i][nt] = lds64(xb_a + 32u * (4 * (ch * rows_per + w) + i - 1) + nt * 8 * xstride);
+                }
             }
-        }
-    }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int ch = 0; ch < CH; ++ch) {
+                const uint32_t prev = __funnelshift_r(wm1[ch][i], w0[ch][i], pos[ch][i]);
+                const uint32_t lo = __funnelshift_r(w0[ch][i], w1[ch][i], pos[ch][i]);
+                if (!(kFirst && i == 0))
+                    finish_block(ch, xb_a + 32u * (4 * (ch * rows_per + w) + i - 1), prev,
+                                 kPreX ? xf[ch][i] : nullptr);
+                d0[ch] = prmt(lo, kFill, e[ch][i]);
+                sel_hi[ch] = e[ch][i] >> 16;
+            }
+    };
+    word(std::true_type{}, 0);
+    for (int w = 1; w < rows_per; ++w) word(std::false_type{}, w);
 #pragma unroll
     for (int ch = 0; ch < CH; ++ch) {
-        const uint32_t* q = payp + ((b8[ch] >> 5) << 5);
-        const uint32_t prev = __funnelshift_r(*(q - 32), q[0], b8[ch]);
-        finish_block(ch, 4 * (ch + 1) * rows_per - 1, prev);
+        const uint32_t a = pay_a + ((b8[ch] >> 5) << 7);
+        const uint32_t prev = __funnelshift_r(lds32(a - 128u), lds32(a), b8[ch]);
+        finish_block(ch, xb_a + 32u * (4 * (ch + 1) * rows_per - 1), prev, nullptr);
     }
 }
 
 // ---- the kernel -----------------------------------------------------------------------------
-template <int NT, int STAGES, int CH>
+// exact floor(u / d) for u < 2^24, d < 2^16, with m = floor(2^40 / d) + 1 precomputed on the host
+__device__ __forceinline__ uint32_t fdiv(uint32_t u, unsigned long long m)
+{
+    return (uint32_t)(((unsigned long long)u * m) >> 40);
+}
+
+// LA = local mode (shared-memory strip accumulators), else direct mode.
+template <int NT, int STAGES, int CH, bool LA>
 __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
-    const uint32_t beg = __ldg(p.cta_begin + blockIdx.x), end = __ldg(p.cta_begin + blockIdx.x + 1);
-    if (beg >= end) return;
+    const bool timing = p.timers != nullptr;
+    long long t_wait = 0, t_decode = 0, t_epi = 0, t_start = timing ? clock64() : 0, t_first = 0;
+    long long dbg[4] = {0, 0, 0, 0};   // prologue checkpoints (cycles since t_start)
+    const unsigned long long g_start = timing ? global_timer_ns() : 0;
 
-    const int xstride = p.K_L + 32;
+    // ---- shared-memory carve-up (mirrored by plan_launch on the host) --------------------------
+    const int xstride = p.G * p.K_L + 32;
     uint32_t* lut = reinterpret_cast<uint32_t*>(smem);
     uint8_t* x8 = smem + kLutBytes;
     int32_t* sx16 = reinterpret_cast<int32_t*>(x8 + NT * 8 * xstride);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sx16 + 64);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sx16 + p.G * NT * 8);
+    uint32_t* claim = reinterpret_cast<uint32_t*>(bars + 32 * STAGES);
+    int32_t* acc_l = reinterpret_cast<int32_t*>(claim + 32);               // [s_local][NT*128]
+    uint32_t* cnt_l = reinterpret_cast<uint32_t*>(acc_l + p.s_local * NT * 128);  // [s_local]
+    uint32_t* off_s = cnt_l + p.s_local;                                    // [kOffTable][2]
     uint8_t* ring0 = reinterpret_cast<uint8_t*>(
-        (reinterpret_cast<uintptr_t>(bars + 32 * STAGES + 16) + 127) & ~uintptr_t(127));
+        (reinterpret_cast<uintptr_t>(off_s + 2 * kOffTable) + 127) & ~uintptr_t(127));
     uint8_t* my_ring = ring0 + (size_t)warp * STAGES * p.slot_bytes;
-    const bool timing = p.timers != nullptr;
-    long long t_wait = 0, t_decode = 0, t_epi = 0, t_start = timing ? clock64() : 0;
 
-    // ---- this warp's tiles: beg + warp, beg + warp + n_warps, ... (static round robin) --------
-    // Start the first copies before anything else: the barriers are private to the warp.
+    // ---- prologue: the latency-critical small loads go out first ------------------------------
+    // With a single K range the activations to stage are known before the CTA's tile range is:
+    // fetch them (into registers) ahead of everything else.
+    constexpr int kXPre = NT == 1 ? 8 : NT == 2 ? 4 : 0;   // 16-byte units of X a thread prefetches
+    const bool x_early = kXPre > 0 && (p.n_segs <= p.G) && p.x_fast == 2;
+    uint4 xpre[kXPre > 0 ? kXPre : 1];
+    const int x_upr = p.K_L / 32, x_total = NT * 8 * p.n_segs * x_upr;
+    if (x_early) {
+        const int64_t ldx = ((int64_t)p.K + 1) / 2;
+#pragma unroll
+        for (int b = 0; b < kXPre; ++b) {
+            const int u = threadIdx.x + b * blockDim.x;
+            xpre[b] = make_uint4(0, 0, 0, 0);
+            if (u < x_total) {
+                const int pi = u / x_upr, q = u - pi * x_upr;
+                const int sgl = pi / (NT * 8), n = pi - sgl * (NT * 8);
+                const int64_t k = (int64_t)sgl * p.K_L + 32 * q;
+                if (n < p.N && k < p.K)
+                    xpre[b] = __ldg(reinterpret_cast<const uint4*>(p.X + (int64_t)n * ldx + k / 2));
+            }
+        }
+    }
+    const uint32_t beg = p.cta_begin[blockIdx.x], end = p.cta_begin[blockIdx.x + 1];
+    if (beg >= end) return;
+#ifndef US_EXP_EPI_TIMERS
+    if (timing) dbg[0] = clock64() - t_start;
+#endif
+
+    // position u of the processing order -> K range, strip, segment within the range, tile index
+    const uint32_t kr_stride = (uint32_t)p.n_strips * (uint32_t)p.G;
+    const int n_kr = (p.n_segs + p.G - 1) / p.G;
+    const int g_last = p.n_segs - (n_kr - 1) * p.G;
+    auto tile_of = [&](uint32_t u, int& kr, int& rb, int& sgl) -> uint32_t {
+        kr = (n_kr == 1) ? 0 : (int)fdiv(u, p.mg_krs);
+        const uint32_t q = u - (uint32_t)kr * kr_stride;
+        const bool lastr = (kr == n_kr - 1);
+        const uint32_t g_kr = lastr ? (uint32_t)g_last : (uint32_t)p.G;
+        rb = (int)fdiv(q, lastr ? p.mg_glast : p.mg_g);
+        sgl = (int)(q - (uint32_t)rb * g_kr);
+        return (uint32_t)rb * (uint32_t)p.n_segs + (uint32_t)(kr * p.G + sgl);
+    };
+
+    // tile index of position u; with a single K range the two orders coincide
+    auto tile_index = [&](uint32_t u) -> uint32_t {
+        if (n_kr == 1) return u;
+        int kr, rb, sgl;
+        return tile_of(u, kr, rb, sgl);
+    };
+
+    // ---- tile queue of this warp: runs of R consecutive positions --------------------------------
+    // The first runs are fixed (run w, w + n_warps, ...: enough to fill the ring and one ahead);
+    // later runs are claimed from the CTA's counter. A run mostly stays inside one strip, so its
+    // partial sums are carried in registers and flushed once.
+    const uint32_t R = (uint32_t)p.run_len;
+    const int n_static = (STAGES + 1 + (int)R - 1) / (int)R;   // fixed runs per warp
+    auto static_pos = [&](int k) -> uint32_t {                 // k-th position of the fixed sequence
+        const uint32_t j = (uint32_t)k / R, i = (uint32_t)k - j * R;
+        return beg + ((uint32_t)warp + j * (uint32_t)n_warps) * R + i;
+    };
+    uint32_t run_next = 0, run_end = 0;   // the run being handed out (after the fixed positions)
+    int static_k = STAGES + 1;            // fixed positions already handed out
+    auto next_pos = [&]() -> uint32_t {
+        if (static_k < n_static * (int)R) return static_pos(static_k++);
+        if (run_next == run_end) {
+            uint32_t b = 0;
+            if (lane == 0) b = atomicAdd(claim, R);
+            run_next = __shfl_sync(0xffffffffu, b, 0);
+            run_end = run_next + R;
+        }
+        return run_next++;
+    };
+
+    // ---- start the first copies: the barriers are private to the warp ---------------------------
     if (lane == 0) {
 #pragma unroll
         for (int s = 0; s < STAGES; ++s) mbar_init(smem_u32(&bars[warp * STAGES + s]), 1);
@@ -288,32 +465,64 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncwarp();
-    uint32_t next_issue = beg + warp;  // next tile to start a copy for
-    uint32_t next_proc = beg + warp;   // next tile to decode
-    uint32_t po0 = 0, po1 = 0;         // offsets of tile next_issue (valid in lane 0)
+    uint32_t item[STAGES];        // position u held (or awaited) by each ring slot
+    uint32_t ahead;               // next position, whose offsets are already being fetched
+    uint32_t po0 = 0, po1 = 0;    // its offsets (valid in lane 0)
     {
-        // lanes 0..STAGES fetch the offsets of the first STAGES+1 tiles in parallel
+        // lanes 0..STAGES fetch the offsets of the first STAGES+1 positions in parallel
+        const uint32_t mine = static_pos(lane <= STAGES ? lane : 0);
         uint32_t o0 = 0, o1 = 0;
-        const uint32_t mine = next_issue + (uint32_t)lane * (uint32_t)n_warps;
-        if (lane <= STAGES && mine < end) { o0 = __ldg(p.item_off + mine); o1 = __ldg(p.item_off + mine + 1); }
+        if (lane <= STAGES && mine < end) {
+            const uint32_t t = tile_index(mine);
+            o0 = __ldg(p.item_off + t); o1 = __ldg(p.item_off + t + 1);
+        }
+        // meanwhile the CTA fetches the offsets of its first kOffTable positions into shared
+        // memory (visible after the first __syncthreads); later refills never wait on DRAM
+        for (int i = threadIdx.x; i < kOffTable; i += blockDim.x) {
+            const uint32_t u = beg + (uint32_t)i;
+            if (u < end) {
+                const uint32_t t = tile_index(u);
+                off_s[2 * i] = __ldg(p.item_off + t);
+                off_s[2 * i + 1] = __ldg(p.item_off + t + 1);
+            }
+        }
+        // (built here: its arithmetic overlaps the offset loads issued just above)
+        // Selector table, replicated once per bank. Every thread computes the entries it needs (pure
+        // register arithmetic: no memory round trip in the prologue) and a warp writes one entry row.
+        for (int e0 = 0; e0 < 256; e0 += blockDim.x) {
+            const int m = e0 + threadIdx.x;
+            const uint32_t mine = m < 256 ? lut_entry(m) : 0u;
+            // thread (w, l) holds entry e0 + 32 w + l; row e0 + 32 w + r is broadcast from lane r
+    #pragma unroll 4
+            for (int r = 0; r < 32; ++r) {
+                const uint32_t v = __shfl_sync(0xffffffffu, mine, r);
+                const int e = e0 + 32 * warp + r;
+                if (e < 256) lut[e * 32 + lane] = v;
+            }
+        }
 #pragma unroll
         for (int s = 0; s <= STAGES; ++s) {
             const uint32_t a = __shfl_sync(0xffffffffu, o0, s), b = __shfl_sync(0xffffffffu, o1, s);
+            const uint32_t u = static_pos(s);
             if (s < STAGES) {
-                if (next_issue < end && lane == 0) {
+                item[s] = u;
+                if (u < end && lane == 0) {
                     const uint32_t bar = smem_u32(&bars[warp * STAGES + s]);
                     mbar_expect_tx(bar, (b - a) * 16u);
                     bulk_g2s(smem_u32(my_ring + (size_t)s * p.slot_bytes), p.blob + (size_t)a * 16u, (b - a) * 16u, bar);
                 }
-                next_issue += n_warps;
             } else {
-                po0 = a; po1 = b;
+                ahead = u; po0 = a; po1 = b;
             }
         }
     }
-    // refill slot s with tile next_issue (offsets prefetched into po0/po1), then prefetch the next
+#ifndef US_EXP_EPI_TIMERS
+    if (timing) dbg[1] = clock64() - t_start;
+#endif
+    if (threadIdx.x == 0) *claim = beg + (uint32_t)n_static * (uint32_t)n_warps * R;
+    // refill slot s with the position fetched ahead
     auto refill = [&](int s) {
-        if (lane == 0 && next_issue < end) {
+        if (lane == 0 && ahead < end) {
             const uint32_t bytes = (po1 - po0) * 16u;
             const uint32_t bar = smem_u32(&bars[warp * STAGES + s]);
             // the warp's earlier generic-proxy reads of this slot are ordered before the refill
@@ -321,25 +530,36 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
             mbar_expect_tx(bar, bytes);
             bulk_g2s(smem_u32(my_ring + (size_t)s * p.slot_bytes), p.blob + (size_t)po0 * 16u, bytes, bar);
         }
-        next_issue += n_warps;
-        if (lane == 0 && next_issue < end) {
-            po0 = __ldg(p.item_off + next_issue);
-            po1 = __ldg(p.item_off + next_issue + 1);
+        return ahead;
+    };
+    // take the next position and start fetching its offsets (called at the end of a tile's
+    // bookkeeping: a fence issued after these loads would have to wait for them)
+    auto fetch_ahead = [&]() {
+        ahead = next_pos();
+        if (lane == 0 && ahead < end) {
+            const uint32_t i = ahead - beg;
+            if (i < (uint32_t)kOffTable) {
+                po0 = off_s[2 * i]; po1 = off_s[2 * i + 1];
+            } else {
+                const uint32_t t = tile_index(ahead);
+                po0 = __ldg(p.item_off + t); po1 = __ldg(p.item_off + t + 1);
+            }
         }
     };
 
-    // selector table, replicated once per bank
-    for (int e = warp; e < 256; e += n_warps) lut[e * 32 + lane] = c_lut.v[e];
-
     uint32_t phase = 0;   // bit s = parity to wait for on stage s
     bool dead = false;    // a bounded wait ran out: stop working, keep the barriers balanced
-    int pend_rb = -1;     // strip whose split-K contribution is issued but not yet signalled
+    int pend_rb = -1;     // direct mode: strip whose contribution is issued but not yet signalled
+    uint32_t pend_n = 0;  //              and the number of tiles in it
     const int t2 = (lane & 3) * 2;
+    const uint32_t lut_a = smem_u32(lut) + 4u * lane;
 
     // store the 16 x N results of strip rb held in fragment order in v
-    auto store_strip = [&](int rb, int (&v)[NT][4]) {
-        const int g = lane >> 2;
-        const int m_lo = __ldg(p.row_order + rb * 16 + g), m_hi = __ldg(p.row_order + rb * 16 + g + 8);
+    auto store_strip = [&](int rb, int (&v)[NT][4], int m_lo, int m_hi) {
+        if (m_lo == kNoRow) {   // not prefetched by the caller
+            m_lo = __ldg(p.row_order + rb * 16 + (lane >> 2));
+            m_hi = __ldg(p.row_order + rb * 16 + (lane >> 2) + 8);
+        }
         float sw_lo = 0.f, sw_hi = 0.f;
         if (p.fp16_out) {
             if (m_lo >= 0) sw_lo = __half2float(__ushort_as_half(__ldg(p.w_scale + m_lo)));
@@ -362,14 +582,22 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
                 }
             }
     };
-    // announce one finished split-K contribution to strip rb; the last arrival finalizes it
-    auto signal_strip = [&](int rb) {
+    // add v to the global workspace of strip rb
+    auto red_global = [&](int rb, int (&v)[NT][4]) {
+        int32_t* accp = p.acc + (size_t)rb * (NT * 128) + lane;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) atomicAdd(accp + nt * 128 + j * 32, v[nt][j]);
+    };
+    // announce n_tiles finished contributions to strip rb; the arrival that completes it finalizes
+    auto signal_strip = [&](int rb, uint32_t n_tiles, int m_lo, int m_hi) {
         __threadfence();
         __syncwarp();
         uint32_t old = 0;
-        if (lane == 0) old = atomicAdd(p.cnt + rb, 1u);
+        if (lane == 0) old = atomicAdd(p.cnt + rb, n_tiles);
         old = __shfl_sync(0xffffffffu, old, 0);
-        if (old == (uint32_t)p.n_segs - 1) {
+        if (old + n_tiles == (uint32_t)p.n_segs) {
             __threadfence();
             int32_t* accp = p.acc + (size_t)rb * (NT * 128) + lane;
             int v[NT][4];
@@ -381,20 +609,87 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
                     __stcg(accp + nt * 128 + j * 32, 0);
                 }
             if (lane == 0) p.cnt[rb] = 0;
-            store_strip(rb, v);
+            store_strip(rb, v, m_lo, m_hi);
         }
     };
 
-    const int sg_first = beg / p.n_strips, sg_last = (end - 1) / p.n_strips;
+    int kr_first, kr_last, d0_, d1_;
+    tile_of(beg, kr_first, d0_, d1_);
+    tile_of(end - 1, kr_last, d0_, d1_);
     int cur = 0;
-    for (int sg = sg_first; sg <= sg_last; ++sg) {
-        if (sg != sg_first) __syncthreads();  // everyone is done with the previous segment's X
-        stage_x<NT>(p, sg, x8, sx16, warp, lane, n_warps);
-        __syncthreads();
-        const uint32_t seg_base = (uint32_t)sg * (uint32_t)p.n_strips;
-        const uint32_t seg_end = min(end, seg_base + (uint32_t)p.n_strips);
+    int y[NT][4];          // partial Y of the run in flight (fragment order)
+    uint32_t y_n = 0;      // tiles summed in y
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) y[nt][0] = y[nt][1] = y[nt][2] = y[nt][3] = 0;
 
-        while (!dead && next_proc < seg_end) {
+    // Stage the activations of K range kr: clear the sums, expand X, synchronise.
+    auto stage_range = [&](int kr, int g_kr, bool use_prefetched) {
+        for (int i = threadIdx.x; i < p.G * NT * 8; i += blockDim.x) sx16[i] = 0;
+        if (LA) {
+            for (int i = threadIdx.x; i < p.s_local * NT * 128; i += blockDim.x) acc_l[i] = 0;
+            for (int i = threadIdx.x; i < p.s_local; i += blockDim.x) cnt_l[i] = 0;
+        }
+        __syncthreads();
+        if (use_prefetched) {
+            // expand the prefetched units; anything beyond them goes through the general path
+#pragma unroll
+            for (int b = 0; b < kXPre; ++b) {
+                const int u = threadIdx.x + b * blockDim.x;
+                if (u < x_total) {
+                    const int pi = u / x_upr, q = u - pi * x_upr;
+                    const int sgl = pi / (NT * 8), n = pi - sgl * (NT * 8);
+                    int32_t sacc = 0;
+                    uint4 vlo, vhi;
+                    uint2 t;
+                    t = expand8(xpre[b].x, sacc); vlo.x = t.x; vlo.y = t.y;
+                    t = expand8(xpre[b].y, sacc); vlo.z = t.x; vlo.w = t.y;
+                    t = expand8(xpre[b].z, sacc); vhi.x = t.x; vhi.y = t.y;
+                    t = expand8(xpre[b].w, sacc); vhi.z = t.x; vhi.w = t.y;
+                    uint4* dst = reinterpret_cast<uint4*>(x8 + n * xstride + sgl * p.K_L + 32 * q);
+                    dst[0] = vlo; dst[1] = vhi;
+                    if (x_upr == 32) {   // one warp holds exactly one (segment, token) pair
+                        sacc = __reduce_add_sync(0xffffffffu, sacc);
+                        if (lane == 0) sx16[pi] = sacc;
+                    } else if (sacc) {
+                        atomicAdd(sx16 + pi, sacc);
+                    }
+                }
+            }
+            stage_x<NT>(p, 0, g_kr, x8, xstride, sx16, kXPre * (int)blockDim.x);
+        } else {
+            stage_x<NT>(p, kr * p.G, g_kr, x8, xstride, sx16, 0);
+        }
+        __syncthreads();
+    };
+#ifndef US_EXP_EPI_TIMERS
+    if (timing) dbg[2] = clock64() - t_start;
+#endif
+    // The first range is staged here, outside the loop, so that the prefetched X registers are
+    // dead before the decode loop starts.
+    stage_range(kr_first, (kr_first == n_kr - 1) ? g_last : p.G, x_early);
+#ifndef US_EXP_EPI_TIMERS
+    if (timing) dbg[3] = clock64() - t_start;
+#endif
+
+    for (int kr = kr_first; kr <= kr_last; ++kr) {
+        const int g_kr = (kr == n_kr - 1) ? g_last : p.G;
+        const unsigned long long mg = (kr == n_kr - 1) ? p.mg_glast : p.mg_g;
+        const uint32_t base = (uint32_t)kr * kr_stride;
+        const uint32_t lo = max(beg, base), hi = min(end, base + (uint32_t)p.n_strips * (uint32_t)g_kr);
+        const uint32_t qlo = lo - base, qhi = hi - base;
+        const int rb_first = (int)fdiv(qlo, mg);
+        if (kr != kr_first) {
+            __syncthreads();  // everyone is done with the previous range's X and sums
+            stage_range(kr, g_kr, false);
+        }
+        if (timing && t_first == 0) t_first = clock64();
+
+        while (!dead) {
+            uint32_t u = 0;
+#pragma unroll
+            for (int s = 0; s < STAGES; ++s)
+                if (s == cur) u = item[s];
+            if (u >= hi) break;
             const long long t0 = timing ? clock64() : 0;
             const uint32_t bar = smem_u32(&bars[warp * STAGES + cur]);
             if (!mbar_wait_bounded(bar, (phase >> cur) & 1u)) {
@@ -405,69 +700,142 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
             phase ^= 1u << cur;
             const long long t1 = timing ? clock64() : 0;
 
+            const uint32_t q = u - base;
+            const int rb = (int)fdiv(q, mg);
+            const int sgl = (int)(q - (uint32_t)rb * (uint32_t)g_kr);
+            // original rows of this strip's fragment rows g and g + 8: needed only when the strip is
+            // stored, fetched now so that the loads complete behind the decode
+            const int m_lo = __ldg(p.row_order + rb * 16 + (lane >> 2));
+            const int m_hi = __ldg(p.row_order + rb * 16 + (lane >> 2) + 8);
             int c[NT][4];
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0;
-            const uint32_t* slot = reinterpret_cast<const uint32_t*>(my_ring + (size_t)cur * p.slot_bytes);
-            process_tile<NT, CH>(slot, lut, x8, xstride, p.mask_rows, lane, c);
+            const uint32_t slot_a = smem_u32(my_ring + (size_t)cur * p.slot_bytes);
+            const uint32_t xb_a = smem_u32(x8) + (lane >> 2) * xstride + 8 * (lane & 3) + sgl * p.K_L;
+            process_tile<NT, CH>(slot_a, lut_a, xb_a, xstride, p.mask_rows, lane, c);
             __syncwarp();
             const long long t2c = timing ? clock64() : 0;
 
-            refill(cur);  // before the epilogue, so that the copy overlaps it
+#ifdef US_EXP_EPI_TIMERS
+            long long te0 = clock64();
+#endif
+            // refill this slot right away, so that the copy overlaps the bookkeeping
+            {
+                const uint32_t issued = refill(cur);
+#pragma unroll
+                for (int s = 0; s < STAGES; ++s)
+                    if (s == cur) item[s] = issued;
+            }
             cur = (cur + 1 == STAGES) ? 0 : cur + 1;
 
-            // ---- split-K reduce + finalize ----
-            const int rb = (int)(next_proc - seg_base);
-            next_proc += n_warps;
+#ifdef US_EXP_EPI_TIMERS
+            long long te1 = clock64(); dbg[0] += te1 - te0;
+#endif
+            // ---- fragment sums -> partial Y of this tile, added to the run's sums ----
+            const int32_t* sxp = sx16 + sgl * (NT * 8);
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
                 const int n0 = nt * 8 + t2;
-                const int s0 = sx16[n0] >> 4, s1 = sx16[n0 + 1] >> 4;
-                const int e0 = c[nt][2] >> 4, e1 = c[nt][3] >> 4;
-                const int yhi0 = (c[nt][0] - c[nt][2]) >> 8, yhi1 = (c[nt][1] - c[nt][3]) >> 8;  // row g+8
-                c[nt][0] = e0 - 8 * s0; c[nt][1] = e1 - 8 * s1;                                 // row g
-                c[nt][2] = yhi0; c[nt][3] = yhi1;
+                const int s0 = sxp[n0] >> 4, s1 = sxp[n0 + 1] >> 4;
+                y[nt][0] += (c[nt][2] >> 4) - 8 * s0;                 // strip row g
+                y[nt][1] += (c[nt][3] >> 4) - 8 * s1;
+                y[nt][2] += (c[nt][0] - c[nt][2]) >> 8;               // strip row g + 8
+                y[nt][3] += (c[nt][1] - c[nt][3]) >> 8;
             }
-            if (p.n_segs == 1) {
-                store_strip(rb, c);
-            } else {
-                // The previous tile's red.adds were issued a whole tile ago: its fence is cheap now.
-                if (pend_rb >= 0) signal_strip(pend_rb);
-                int32_t* accp = p.acc + (size_t)rb * (NT * 128) + lane;
+            ++y_n;
+            // the run goes on if this warp's next tile is the next segment of the same strip
+            uint32_t u_next = 0;
 #pragma unroll
-                for (int nt = 0; nt < NT; ++nt)
+            for (int s = 0; s < STAGES; ++s)
+                if (s == cur) u_next = item[s];
+            const bool more = (u_next == u + 1u) && (u_next < hi) && (sgl + 1 < g_kr);
+#ifdef US_EXP_EPI_TIMERS
+            long long te2 = clock64(); dbg[1] += te2 - te1;
+#endif
+            if (!more) {
+                if (LA) {
+                    // tiles of this strip inside the CTA's part of the K range
+                    const uint32_t expected = min(qhi, (uint32_t)(rb + 1) * (uint32_t)g_kr) - max(qlo, (uint32_t)rb * (uint32_t)g_kr);
+                    const int sl = rb - rb_first;
+                    if (y_n == expected) {   // the whole of it was summed in registers
+                        if (expected == (uint32_t)p.n_segs) store_strip(rb, y, m_lo, m_hi);
+                        else { red_global(rb, y); signal_strip(rb, expected, m_lo, m_hi); }
+                    } else {
+                        int32_t* al = acc_l + sl * (NT * 128) + lane;
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) atomicAdd(accp + nt * 128 + j * 32, c[nt][j]);
-                pend_rb = rb;
+                        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) atomicAdd(al + nt * 128 + j * 32, y[nt][j]);
+                        __threadfence_block();
+                        __syncwarp();
+                        uint32_t old = 0;
+                        if (lane == 0) old = atomicAdd(cnt_l + sl, y_n);
+                        old = __shfl_sync(0xffffffffu, old, 0);
+                        if (old + y_n == expected) {   // the CTA's last tiles of this strip: flush it
+                            __threadfence_block();
+#pragma unroll
+                            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) y[nt][j] = *(volatile int32_t*)(al + nt * 128 + j * 32);
+                            if (expected == (uint32_t)p.n_segs) store_strip(rb, y, m_lo, m_hi);
+                            else { red_global(rb, y); signal_strip(rb, expected, m_lo, m_hi); }
+                        }
+                    }
+                } else if (p.n_segs == 1) {
+                    store_strip(rb, y, m_lo, m_hi);
+                } else {
+                    // The previous run's red.adds were issued a while ago: its fence is cheap now.
+                    if (pend_rb >= 0) signal_strip(pend_rb, pend_n, kNoRow, kNoRow);
+                    red_global(rb, y);
+                    pend_rb = rb; pend_n = y_n;
+                }
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) y[nt][0] = y[nt][1] = y[nt][2] = y[nt][3] = 0;
+                y_n = 0;
             }
+#ifdef US_EXP_EPI_TIMERS
+            long long te3 = clock64(); dbg[2] += te3 - te2;
+#endif
+            fetch_ahead();
+#ifdef US_EXP_EPI_TIMERS
+            dbg[3] += clock64() - te3;
+#endif
             if (timing) {
                 const long long t3 = clock64();
                 t_wait += t1 - t0; t_decode += t2c - t1; t_epi += t3 - t2c;
             }
         }
     }
-    if (pend_rb >= 0) signal_strip(pend_rb);
+    if (pend_rb >= 0) signal_strip(pend_rb, pend_n, kNoRow, kNoRow);
 
-    // Drain: copies this warp issued but never consumed must land before the CTA exits
-    // (only after a bounded wait ran out; in a normal run every issued tile was consumed).
+    // Drain (only after a bounded wait ran out; in a normal run every issued tile was consumed):
+    // copies this warp issued must land before the CTA exits.
     if (dead) {
-        uint32_t it = next_proc;
 #pragma unroll
         for (int s = 0; s < STAGES; ++s) {
-            if (it < end && it < next_issue) {
-                const uint32_t bar = smem_u32(&bars[warp * STAGES + cur]);
-                if (!mbar_wait_bounded(bar, (phase >> cur) & 1u) && lane == 0) atomicExch(p.err, kErrTimeout);
+            if (item[s] < end) {
+                const uint32_t bar = smem_u32(&bars[warp * STAGES + s]);
+                if (!mbar_wait_bounded(bar, (phase >> s) & 1u) && lane == 0) atomicExch(p.err, kErrTimeout);
             }
-            it += n_warps;
-            cur = (cur + 1 == STAGES) ? 0 : cur + 1;
         }
     }
     if (timing && lane == 0) {
+        const long long t_end = clock64();
         atomicAdd(p.timers + 0, (unsigned long long)t_wait);
         atomicAdd(p.timers + 1, (unsigned long long)t_decode);
         atomicAdd(p.timers + 2, (unsigned long long)t_epi);
-        atomicAdd(p.timers + 3, (unsigned long long)(clock64() - t_start));
+        atomicAdd(p.timers + 3, (unsigned long long)(t_end - t_start));
         atomicAdd(p.timers + 4, 1ull);
+        atomicAdd(p.timers + 5, (unsigned long long)(t_first - t_start));
+        atomicMax(p.timers + 6, (unsigned long long)(t_end - t_start));
+        atomicMin(p.timers + 7, g_start);
+        atomicMax(p.timers + 8, (unsigned long long)global_timer_ns());
+        for (int i = 0; i < 4; ++i) atomicAdd(p.timers + 9 + i, (unsigned long long)dbg[i]);
+        // per-CTA sums: warp lifetimes, waits, decode; and the CTA's start offset from the first one
+        atomicAdd(p.timers + 16 + 4 * blockIdx.x + 0, (unsigned long long)(t_end - t_start));
+        atomicAdd(p.timers + 16 + 4 * blockIdx.x + 1, (unsigned long long)t_wait);
+        atomicAdd(p.timers + 16 + 4 * blockIdx.x + 2, (unsigned long long)t_decode);
+        if (warp == 0) p.timers[16 + 4 * blockIdx.x + 3] = g_start;
     }
 }
 
