@@ -432,6 +432,7 @@ def run_only(args):
         sw.check()
     t = e0.elapsed_time(e1) * 1e-3 / (args.steps * len(case.sw))
     alg = algorithmic_bytes(case.stats, N, fp16)
+    t_graph = case.time_passes(N, fp16, passes=max(3, args.steps), warmup=3)
     # one more pass with the kernel's stage timers on (not part of the timing above)
     for sw in case.sw:
         binding.us_stage_timers(sw.handle, 1)
@@ -443,7 +444,8 @@ def run_only(args):
             tm[k] = tm.get(k, 0) + v
     per_warp = ("wait", "decode", "epilogue", "lifetime", "prologue")
     timers = {k: (v / tm["warps"] if k in per_warp else v / len(case.sw)) for k, v in tm.items()}
-    print(json.dumps({"only": args.only, "us_per_launch_stream_order": t * 1e6, "alg_bytes": alg,
+    print(json.dumps({"only": args.only, "us_per_launch_graph": t_graph * 1e6, "gbs_graph": alg / t_graph / 1e9,
+                      "us_per_launch_stream_order": t * 1e6, "alg_bytes": alg,
                       "stored_bytes": binding.us_spmm_bytes(case.sw[0].handle, N, fp16),
                       "gbs": alg / t / 1e9, "replicas": len(case.sw), "format": list(case.stats["fmt"]),
                       "launch": binding.us_launch_info(case.sw[0].handle, N),

@@ -295,9 +295,11 @@ us_status us_spmm(us_handle* h, const void* X, int32_t N, const void* x_scale, v
         p.mg_g = magic((uint64_t)p.G);
         p.mg_glast = magic((uint64_t)g_last);
         p.mg_krs = magic((uint64_t)hm.n_strips * (uint64_t)p.G);
-        // claim runs of up to half a strip's segments of the range, so that a CTA's warps still
-        // share its strips evenly
-        const int want = run_knob() > 0 ? run_knob() : std::max(1, p.G / 2);
+        // Claim runs of up to half a strip's segments of the range (the partial sums of a run stay
+        // in registers), but never so long that a CTA's warps run out of runs to share.
+        const int64_t per_cta = std::max<int64_t>(1, hm.n_items / std::max(1, h->sm_count));
+        const int balanced = (int)std::max<int64_t>(1, per_cta / (4 * (int64_t)g.warps));
+        const int want = run_knob() > 0 ? run_knob() : std::min(std::max(1, p.G / 2), balanced);
         p.run_len = std::max(1, std::min(want, p.G));
     }
     p.row_order = h->d_row_order; p.w_scale = h->d_w_scale;

@@ -261,10 +261,50 @@ __device__ __forceinline__ void stage_x(const SpmmParams& p, int seg0, int n_seg
     }
 }
 
+// Store the 16 x N results held in fragment order in v: fragment rows g -> original row m_lo,
+// rows g + 8 -> m_hi (negative = padding row), with the optional fp16 dequantisation.
+struct StoreCtx {   // what the store needs, by value (the full parameter block is large)
+    void* Y;
+    const uint16_t* w_scale;
+    const uint16_t* x_scale;
+    int32_t* acc;
+    uint32_t* cnt;
+    int32_t M, N, fp16_out;
+};
+template <int NT>
+__device__ __forceinline__ void store_rows(const StoreCtx p, const int (&v)[NT][4], int lane, int m_lo, int m_hi)
+{
+    const int t2 = (lane & 3) * 2;
+    float sw_lo = 0.f, sw_hi = 0.f;
+    if (p.fp16_out) {
+        if (m_lo >= 0) sw_lo = __half2float(__ushort_as_half(__ldg(p.w_scale + m_lo)));
+        if (m_hi >= 0) sw_hi = __half2float(__ushort_as_half(__ldg(p.w_scale + m_hi)));
+    }
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int n = nt * 8 + t2 + (j & 1);
+            const int m = (j < 2) ? m_lo : m_hi;
+            if (n >= p.N || m < 0) continue;
+            const size_t o = (size_t)n * p.M + m;
+            if (p.fp16_out) {
+                const float sx = __half2float(__ushort_as_half(__ldg(p.x_scale + n)));
+                const float r = (float)v[nt][j] * ((j < 2) ? sw_lo : sw_hi) * sx;
+                reinterpret_cast<__half*>(p.Y)[o] = __float2half_rn(r);
+            } else {
+                reinterpret_cast<int32_t*>(p.Y)[o] = v[nt][j];
+            }
+        }
+}
+
 // ---- decode + MMA over one staged tile -------------------------------------------------------
-// CH independent decode chains walk consecutive ranges of the tile's k-blocks (chain ch starts at
-// the lane-stream position given by the popcount of the mask words before its range); the chains
-// only share the accumulators, so their shared-memory and permute latencies overlap.
+// One mask word = four k-blocks of the lane. The stream positions of all four (and of the next
+// word's first) follow from the mask word alone, so every shared-memory load of the word is
+// issued before any is used. Block i takes its first four fragment bytes from the window that
+// STARTS at pos[i] and its last four from the window that ENDS at pos[i+1]; the window at
+// pos[4] is carried to the next word, so each word is self-contained (no peeled first or last).
+// CH independent chains walk consecutive ranges of the tile's mask words.
 // All addresses are 32-bit shared-memory addresses: slot_a = the staged tile, lut_a = selector
 // table + 4*lane, xb_a = this lane's first B-fragment of the tile's segment.
 template <int NT, int CH>
@@ -274,8 +314,9 @@ __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, ui
     const int rows_per = mask_rows / CH;
     const uint32_t mask_a = slot_a + 4u * lane;
     const uint32_t pay_a = slot_a + 128u * mask_rows + 4u * lane;
-    uint32_t b8[CH];   // 8 * (byte position in the lane's payload stream), per chain
-    uint32_t d0[CH], sel_hi[CH];
+    constexpr bool kPreX = NT <= 2;   // small N: fetch the X fragments together with the windows
+    uint32_t b8[CH];       // 8 * (byte position in the lane's payload stream), per chain
+    uint32_t cw0[CH], cw1[CH];   // carried window: the two words at / after the chain's position
     b8[0] = 0;
 #pragma unroll
     for (int ch = 1; ch < CH; ++ch) {
@@ -284,23 +325,12 @@ __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, ui
         b8[ch] = b8[ch - 1] + 8u * n;
     }
 #pragma unroll
-    for (int ch = 0; ch < CH; ++ch) d0[ch] = sel_hi[ch] = 0;
-
-    // finish k-block: second permute (mask bits 4..7), low-nibble rows, MMA against its X fragment
-    auto finish_block = [&](int ch, uint32_t xk_a, uint32_t prev, const uint2* xpre) {
-        const uint32_t d1 = prmt(prev, kFill, sel_hi[ch]);
-        const uint32_t e0 = d0[ch] & 0x0F0F0F0Fu, e1 = d1 & 0x0F0F0F0Fu;
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-            const uint2 b = xpre ? xpre[nt] : lds64(xk_a + nt * 8 * xstride);
-            mma_s8(c[nt], d0[ch], e0, d1, e1, b.x, b.y);
-        }
-    };
-    constexpr bool kPreX = NT <= 2;   // small N: fetch the X fragments together with the windows
-    // One mask word = four k-blocks per chain. The stream positions of all four follow from the
-    // mask word alone, so every shared-memory load of the word is issued before any is used.
-    auto word = [&](auto first, int w) {
-        constexpr bool kFirst = decltype(first)::value;
+    for (int ch = 0; ch < CH; ++ch) {
+        const uint32_t a = pay_a + ((b8[ch] >> 5) << 7);
+        cw0[ch] = lds32(a);
+        cw1[ch] = lds32(a + 128u);
+    }
+    for (int w = 0; w < rows_per; ++w) {
         uint32_t pos[CH][5], wm1[CH][4], w0[CH][4], w1[CH][4], e[CH][4];
         uint2 xf[CH][4][kPreX ? NT : 1];
 #pragma unroll
@@ -319,38 +349,58 @@ __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, ui
         for (int i = 0; i < 4; ++i)
 #pragma unroll
             for (int ch = 0; ch < CH; ++ch) {
-                const uint32_t a = pay_a + ((pos[ch][i] >> 5) << 7);
+                const uint32_t a = pay_a + ((pos[ch][i + 1] >> 5) << 7);   // window at the block's END
                 wm1[ch][i] = lds32(a - 128u);
                 w0[ch][i] = lds32(a);
                 w1[ch][i] = lds32(a + 128u);
                 e[ch][i] = lds32(e[ch][i]);
-                if (kPreX && !(kFirst && i == 0)) {
+                if (kPreX) {
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt)
-                        xf[ch][i][nt] = lds64(xb_a + 32u * (4 * (ch * rows_per + w) + i - 1) + nt * 8 * xstride);
+                        xf[ch][i][nt] = lds64(xb_a + 32u * (4 * (ch * rows_per + w) + i) + nt * 8 * xstride);
                 }
             }
 #pragma unroll
         for (int i = 0; i < 4; ++i)
 #pragma unroll
             for (int ch = 0; ch < CH; ++ch) {
-                const uint32_t prev = __funnelshift_r(wm1[ch][i], w0[ch][i], pos[ch][i]);
-                const uint32_t lo = __funnelshift_r(w0[ch][i], w1[ch][i], pos[ch][i]);
-                if (!(kFirst && i == 0))
-                    finish_block(ch, xb_a + 32u * (4 * (ch * rows_per + w) + i - 1), prev,
-                                 kPreX ? xf[ch][i] : nullptr);
-                d0[ch] = prmt(lo, kFill, e[ch][i]);
-                sel_hi[ch] = e[ch][i] >> 16;
-            }
-    };
-    word(std::true_type{}, 0);
-    for (int w = 1; w < rows_per; ++w) word(std::false_type{}, w);
+                // first four bytes: the window starting at pos[i] (carried, or the previous block's)
+                const uint32_t s0 = (i == 0) ? cw0[ch] : w0[ch][i - 1];
+                const uint32_t s1 = (i == 0) ? cw1[ch] : w1[ch][i - 1];
+                const uint32_t lo = __funnelshift_r(s0, s1, pos[ch][i]);
+                const uint32_t prev = __funnelshift_r(wm1[ch][i], w0[ch][i], pos[ch][i + 1]);
+                const uint32_t d0 = prmt(lo, kFill, e[ch][i]);
+                const uint32_t d1 = prmt(prev, kFill, e[ch][i] >> 16);
+                const uint32_t e0 = d0 & 0x0F0F0F0Fu, e1 = d1 & 0x0F0F0F0Fu;
 #pragma unroll
-    for (int ch = 0; ch < CH; ++ch) {
-        const uint32_t a = pay_a + ((b8[ch] >> 5) << 7);
-        const uint32_t prev = __funnelshift_r(lds32(a - 128u), lds32(a), b8[ch]);
-        finish_block(ch, xb_a + 32u * (4 * (ch + 1) * rows_per - 1), prev, nullptr);
+                for (int nt = 0; nt < NT; ++nt) {
+                    const uint2 b = kPreX ? xf[ch][i][nt]
+                                          : lds64(xb_a + 32u * (4 * (ch * rows_per + w) + i) + nt * 8 * xstride);
+                    mma_s8(c[nt], d0, e0, d1, e1, b.x, b.y);
+                }
+            }
+#pragma unroll
+        for (int ch = 0; ch < CH; ++ch) { cw0[ch] = w0[ch][3]; cw1[ch] = w1[ch][3]; }
     }
+}
+
+// Last arrival of a strip in the global workspace: read the sums, leave workspace and counter
+// zeroed, dequantise and store. Kept out of line: it runs once per strip at most, and the decode
+// loop's code should stay small enough for the instruction cache.
+template <int NT>
+__device__ __noinline__ void finalize_strip(const StoreCtx p, int rb, int lane, int m_lo, int m_hi)
+{
+    int32_t* accp = p.acc + (size_t)rb * (NT * 128) + lane;
+    int v[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            v[nt][j] = __ldcg(accp + nt * 128 + j * 32);
+            __stcg(accp + nt * 128 + j * 32, 0);
+        }
+    if (lane == 0) p.cnt[rb] = 0;
+    store_rows<NT>(p, v, lane, m_lo, m_hi);
 }
 
 // ---- the kernel -----------------------------------------------------------------------------
@@ -554,33 +604,13 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
     const int t2 = (lane & 3) * 2;
     const uint32_t lut_a = smem_u32(lut) + 4u * lane;
 
-    // store the 16 x N results of strip rb held in fragment order in v
+    const StoreCtx sctx{p.Y, p.w_scale, p.x_scale, p.acc, p.cnt, p.M, p.N, p.fp16_out};
     auto store_strip = [&](int rb, int (&v)[NT][4], int m_lo, int m_hi) {
         if (m_lo == kNoRow) {   // not prefetched by the caller
             m_lo = __ldg(p.row_order + rb * 16 + (lane >> 2));
             m_hi = __ldg(p.row_order + rb * 16 + (lane >> 2) + 8);
         }
-        float sw_lo = 0.f, sw_hi = 0.f;
-        if (p.fp16_out) {
-            if (m_lo >= 0) sw_lo = __half2float(__ushort_as_half(__ldg(p.w_scale + m_lo)));
-            if (m_hi >= 0) sw_hi = __half2float(__ushort_as_half(__ldg(p.w_scale + m_hi)));
-        }
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int n = nt * 8 + t2 + (j & 1);
-                const int m = (j < 2) ? m_lo : m_hi;
-                if (n >= p.N || m < 0) continue;
-                const size_t o = (size_t)n * p.M + m;
-                if (p.fp16_out) {
-                    const float sx = __half2float(__ushort_as_half(__ldg(p.x_scale + n)));
-                    const float r = (float)v[nt][j] * ((j < 2) ? sw_lo : sw_hi) * sx;
-                    reinterpret_cast<__half*>(p.Y)[o] = __float2half_rn(r);
-                } else {
-                    reinterpret_cast<int32_t*>(p.Y)[o] = v[nt][j];
-                }
-            }
+        store_rows<NT>(sctx, v, lane, m_lo, m_hi);
     };
     // add v to the global workspace of strip rb
     auto red_global = [&](int rb, int (&v)[NT][4]) {
@@ -599,17 +629,11 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
         old = __shfl_sync(0xffffffffu, old, 0);
         if (old + n_tiles == (uint32_t)p.n_segs) {
             __threadfence();
-            int32_t* accp = p.acc + (size_t)rb * (NT * 128) + lane;
-            int v[NT][4];
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    v[nt][j] = __ldcg(accp + nt * 128 + j * 32);
-                    __stcg(accp + nt * 128 + j * 32, 0);
-                }
-            if (lane == 0) p.cnt[rb] = 0;
-            store_strip(rb, v, m_lo, m_hi);
+            if (m_lo == kNoRow) {
+                m_lo = __ldg(p.row_order + rb * 16 + (lane >> 2));
+                m_hi = __ldg(p.row_order + rb * 16 + (lane >> 2) + 8);
+            }
+            finalize_strip<NT>(sctx, rb, lane, m_lo, m_hi);
         }
     };
 
@@ -753,15 +777,16 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
             long long te2 = clock64(); dbg[1] += te2 - te1;
 #endif
             if (!more) {
+                // what happens to the run's sums: 0 = nothing more, 1 = store (the strip is complete
+                // here), 2 = add to the global workspace and announce `tell` tiles
+                int action = 0;
+                uint32_t tell = 0;
                 if (LA) {
                     // tiles of this strip inside the CTA's part of the K range
                     const uint32_t expected = min(qhi, (uint32_t)(rb + 1) * (uint32_t)g_kr) - max(qlo, (uint32_t)rb * (uint32_t)g_kr);
-                    const int sl = rb - rb_first;
-                    if (y_n == expected) {   // the whole of it was summed in registers
-                        if (expected == (uint32_t)p.n_segs) store_strip(rb, y, m_lo, m_hi);
-                        else { red_global(rb, y); signal_strip(rb, expected, m_lo, m_hi); }
-                    } else {
-                        int32_t* al = acc_l + sl * (NT * 128) + lane;
+                    bool flush = (y_n == expected);   // the whole of it was summed in registers
+                    if (!flush) {
+                        int32_t* al = acc_l + (rb - rb_first) * (NT * 128) + lane;
 #pragma unroll
                         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
@@ -769,7 +794,7 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
                         __threadfence_block();
                         __syncwarp();
                         uint32_t old = 0;
-                        if (lane == 0) old = atomicAdd(cnt_l + sl, y_n);
+                        if (lane == 0) old = atomicAdd(cnt_l + (rb - rb_first), y_n);
                         old = __shfl_sync(0xffffffffu, old, 0);
                         if (old + y_n == expected) {   // the CTA's last tiles of this strip: flush it
                             __threadfence_block();
@@ -777,17 +802,23 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
                             for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
                                 for (int j = 0; j < 4; ++j) y[nt][j] = *(volatile int32_t*)(al + nt * 128 + j * 32);
-                            if (expected == (uint32_t)p.n_segs) store_strip(rb, y, m_lo, m_hi);
-                            else { red_global(rb, y); signal_strip(rb, expected, m_lo, m_hi); }
+                            flush = true;
                         }
                     }
+                    if (flush) { action = (expected == (uint32_t)p.n_segs) ? 1 : 2; tell = expected; }
                 } else if (p.n_segs == 1) {
-                    store_strip(rb, y, m_lo, m_hi);
+                    action = 1;
                 } else {
                     // The previous run's red.adds were issued a while ago: its fence is cheap now.
                     if (pend_rb >= 0) signal_strip(pend_rb, pend_n, kNoRow, kNoRow);
                     red_global(rb, y);
                     pend_rb = rb; pend_n = y_n;
+                }
+                if (action == 1) {
+                    store_strip(rb, y, m_lo, m_hi);
+                } else if (action == 2) {
+                    red_global(rb, y);
+                    signal_strip(rb, tell, m_lo, m_hi);
                 }
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) y[nt][0] = y[nt][1] = y[nt][2] = y[nt][3] = 0;
