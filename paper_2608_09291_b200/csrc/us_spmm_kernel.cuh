@@ -168,6 +168,15 @@ __device__ __forceinline__ uint32_t lds32(uint32_t a)
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
     return v;
 }
+// load at a compile-time byte offset from a: the offset goes into the instruction's immediate field
+// instead of costing an integer add per load
+template <int OFF>
+__device__ __forceinline__ uint32_t lds32_at(uint32_t a)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(a), "n"(OFF));
+    return v;
+}
 __device__ __forceinline__ uint2 lds64(uint32_t a)
 {
     uint2 v;
@@ -327,8 +336,8 @@ __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, ui
 #pragma unroll
     for (int ch = 0; ch < CH; ++ch) {
         const uint32_t a = pay_a + ((b8[ch] >> 5) << 7);
-        cw0[ch] = lds32(a);
-        cw1[ch] = lds32(a + 128u);
+        cw0[ch] = lds32_at<0>(a);
+        cw1[ch] = lds32_at<128>(a);
     }
     for (int w = 0; w < rows_per; ++w) {
         uint32_t pos[CH][5], wm1[CH][4], w0[CH][4], w1[CH][4], e[CH][4];
@@ -350,9 +359,9 @@ __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, ui
 #pragma unroll
             for (int ch = 0; ch < CH; ++ch) {
                 const uint32_t a = pay_a + ((pos[ch][i + 1] >> 5) << 7);   // window at the block's END
-                wm1[ch][i] = lds32(a - 128u);
-                w0[ch][i] = lds32(a);
-                w1[ch][i] = lds32(a + 128u);
+                wm1[ch][i] = lds32_at<-128>(a);
+                w0[ch][i] = lds32_at<0>(a);
+                w1[ch][i] = lds32_at<128>(a);
                 e[ch][i] = lds32(e[ch][i]);
                 if (kPreX) {
 #pragma unroll
