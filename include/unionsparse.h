@@ -27,7 +27,9 @@ typedef enum us_status {
     US_ERR_UNSUPPORTED = 4,   /* a valid IE-BME format no kernel of this library implements */
     US_ERR_ALLOC = 5,         /* host or device allocation failed                           */
     US_ERR_CUDA = 6,          /* a CUDA runtime call failed (see us_last_error)             */
-    US_ERR_DEVICE_TIMEOUT = 7 /* a bounded wait inside a kernel gave up (no hang, no trap)  */
+    US_ERR_DEVICE_TIMEOUT = 7,/* a bounded wait inside a kernel gave up (no hang, no trap)  */
+    US_ERR_SCRATCH_TOO_SMALL = 8 /* us_spmm_static_scratch: the problem needs more scratch than
+                                    the library's fixed device array holds                   */
 } us_status;
 
 /*
@@ -112,6 +114,34 @@ us_status us_get_row_order(const us_handle* h, int32_t* perm_out);
  */
 us_status us_spmm(us_handle* h, const void* X, int32_t N, const void* x_scale, void* Y,
                   void* stream);
+
+/*
+ * The same SpMM as us_spmm for callers that must not allocate device memory around the call.
+ * (The paper has no counterpart: this entry point exists for the integration, not the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc / cudaFree are off limits or too costly -- a
+ * serving loop that has handed all device memory to its own pool, a latency-critical path that
+ * cannot afford the device-wide synchronisation an allocation may cause, or a section of a
+ * program in which allocation calls are not permitted. us_spmm keeps its split-K workspace and
+ * arrival counters in memory that the handle allocated; this call instead uses a fixed array that
+ * is part of the library image itself, US_STATIC_SCRATCH_BYTES (4 MiB) per GPU, held by every GPU
+ * that loads the library until the process exits. It calls no allocation routine of any kind.
+ *
+ * Arguments, layouts, output and error behaviour are those of us_spmm, plus:
+ *   - the problem must fit the array: n_strips * (n_tiles_N * 512 + 4) bytes, n_strips =
+ *     ceil(M/16), n_tiles_N = 1, 2, 4, 8 for N <= 8, 16, 32, 64; otherwise
+ *     US_ERR_SCRATCH_TOO_SMALL is returned and nothing is enqueued;
+ *   - the handle's device must be the current device (US_ERR_INVALID_ARG otherwise);
+ *   - the array is shared by every call on that GPU and keeps whatever the last call left in it:
+ *     each call first enqueues a clear of the part it uses on `stream`, then the kernel. Two
+ *     calls that can overlap on the GPU (different streams, no dependency) race on the array and
+ *     give wrong results: serialise them;
+ *   - the first call on a device looks up the array's device address (once per device, with that
+ *     device current). Make that first call before any stream capture begins.
+ */
+#define US_STATIC_SCRATCH_BYTES (4u << 20)
+us_status us_spmm_static_scratch(us_handle* h, const void* X, int32_t N, const void* x_scale, void* Y,
+                                 void* stream);
 
 /*
  * Synchronises the device, then reports the first failure recorded for this handle: a CUDA

@@ -21,7 +21,7 @@ US_OK = 0
 US_ENCODE_HOST_ONLY = 1
 US_ENCODE_SORT_ROWS = 2
 
-EXPORTS = ["us_encode", "us_get_stats", "us_decode", "us_get_row_order", "us_spmm",
+EXPORTS = ["us_encode", "us_get_stats", "us_decode", "us_get_row_order", "us_spmm", "us_spmm_static_scratch",
            "us_last_error", "us_stage_timers", "us_destroy", "us_spmm_bytes", "us_launch_info", "us_status_string"]
 
 
@@ -45,6 +45,7 @@ _lib.us_decode.argtypes = [_vp, _vp]
 _lib.us_get_row_order.argtypes = [_vp, _vp]
 _lib.us_spmm.argtypes = [_vp, _vp, ctypes.c_int32, _vp, _vp, _vp]
 _lib.us_last_error.argtypes = [_vp]
+_lib.us_spmm_static_scratch.argtypes = [_vp, _vp, ctypes.c_int32, _vp, _vp, _vp]
 _lib.us_destroy.argtypes = [_vp]
 _lib.us_stage_timers.argtypes = [_vp, ctypes.c_int32, _vp]
 _lib.us_spmm_bytes.argtypes = [_vp, ctypes.c_int32, ctypes.c_int32]
@@ -112,6 +113,20 @@ def us_get_row_order(h: int) -> np.ndarray:
 def us_spmm(h: int, X_ptr: int, N: int, x_scale_ptr: int | None, Y_ptr: int, stream: int | None = None):
     """Raw call: device pointers as integers, stream as a cudaStream_t integer (None = default)."""
     _check(_lib.us_spmm(h, X_ptr, int(N), x_scale_ptr, Y_ptr, stream), "us_spmm")
+
+
+US_STATIC_SCRATCH_BYTES = 4 << 20
+US_ERR_SCRATCH_TOO_SMALL = 8
+
+
+def us_spmm_static_scratch(h: int, X_ptr: int, N: int, x_scale_ptr: int | None, Y_ptr: int,
+                           stream: int | None = None):
+    """us_spmm for callers that may not allocate device memory around the call: the kernel's
+    scratch (strip sums and arrival counters) is a fixed 4 MiB array inside the library image,
+    shared by all calls on the GPU -- overlapping calls race, and a problem that does not fit
+    is refused with status US_ERR_SCRATCH_TOO_SMALL. Same arguments as us_spmm."""
+    _check(_lib.us_spmm_static_scratch(h, X_ptr, int(N), x_scale_ptr, Y_ptr, stream),
+           "us_spmm_static_scratch")
 
 
 def us_last_error(h: int) -> int:

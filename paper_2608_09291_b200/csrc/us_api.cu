@@ -326,6 +326,88 @@ us_status us_spmm(us_handle* h, const void* X, int32_t N, const void* x_scale, v
     return US_OK;
 }
 
+// ---- us_spmm_static_scratch: the SpMM with its scratch in a fixed device array ------------------
+// The array lives in the library image: every GPU that loads the library holds it until exit.
+// In host code `g_static_scratch` is only a stand-in for the symbol; the device address is looked
+// up once per device with cudaGetSymbolAddress and that pointer is what the kernel receives.
+static __device__ __align__(256) unsigned char g_static_scratch[US_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_scratch_addr[kMaxDevices] = {nullptr};
+}  // namespace
+
+us_status us_spmm_static_scratch(us_handle* h, const void* X, int32_t N, const void* x_scale, void* Y,
+                                 void* stream)
+{
+    if (!h || !X || !Y || N < 1 || N > h->max_N) return US_ERR_INVALID_ARG;
+    if (!h->on_device) return US_ERR_UNSUPPORTED;
+    if (x_scale && !h->d_w_scale) return US_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(X) % 16) return US_ERR_INVALID_ARG;
+    LaunchGeom g;
+    if (!plan_launch(h, N, &g)) return US_ERR_UNSUPPORTED;
+
+    const us::HostMatrix& hm = h->host;
+    // scratch the kernel needs: INT32 strip sums, then one arrival counter per strip
+    const size_t acc_bytes = (size_t)hm.n_strips * g.nt * 128 * sizeof(int32_t);
+    const size_t cnt_bytes = (size_t)hm.n_strips * sizeof(uint32_t);
+    if (acc_bytes + cnt_bytes > (size_t)US_STATIC_SCRATCH_BYTES) return US_ERR_SCRATCH_TOO_SMALL;
+
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return US_ERR_CUDA;
+    if (dev != h->device || dev < 0 || dev >= kMaxDevices) return US_ERR_INVALID_ARG;
+    if (!g_scratch_addr[dev]) {  // set-up, once per device, with that device current
+        void* ptr = nullptr;
+        const cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess || !ptr) { h->sticky = e; return US_ERR_CUDA; }
+        g_scratch_addr[dev] = ptr;
+    }
+    unsigned char* scratch = static_cast<unsigned char*>(g_scratch_addr[dev]);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // The array keeps the previous call's contents: sums and counters must start at zero.
+    cudaError_t e = cudaMemsetAsync(scratch, 0, acc_bytes + cnt_bytes, st);
+    if (e != cudaSuccess) { h->sticky = e; return US_ERR_CUDA; }
+
+    us::SpmmParams p;
+    p.blob = h->d_blob; p.item_off = h->d_item_off;
+    std::memcpy(p.cta_begin, h->cta_begin[g.cls].data(), h->cta_begin[g.cls].size() * sizeof(uint32_t));
+    p.G = h->G[g.cls]; p.s_local = h->s_local[g.cls];
+    {
+        const int64_t n_kr = (hm.n_segs + p.G - 1) / p.G;
+        const int64_t g_last = hm.n_segs - (n_kr - 1) * p.G;
+        auto magic = [](uint64_t d) { return ((1ull << 40) / d) + 1ull; };
+        p.mg_g = magic((uint64_t)p.G);
+        p.mg_glast = magic((uint64_t)g_last);
+        p.mg_krs = magic((uint64_t)hm.n_strips * (uint64_t)p.G);
+        const int64_t per_cta = std::max<int64_t>(1, hm.n_items / std::max(1, h->sm_count));
+        const int balanced = (int)std::max<int64_t>(1, per_cta / (4 * (int64_t)g.warps));
+        const int want = run_knob() > 0 ? run_knob() : std::min(std::max(1, p.G / 2), balanced);
+        p.run_len = std::max(1, std::min(want, p.G));
+    }
+    p.row_order = h->d_row_order; p.w_scale = h->d_w_scale;
+    p.X = static_cast<const uint8_t*>(X);
+    p.x_scale = static_cast<const uint16_t*>(x_scale);
+    p.Y = Y;
+    p.acc = reinterpret_cast<int32_t*>(scratch);
+    p.cnt = reinterpret_cast<uint32_t*>(scratch + acc_bytes);
+    p.err = h->d_err;
+    p.timers = nullptr;
+    p.M = (int32_t)hm.M; p.K = (int32_t)hm.K; p.N = N;
+    p.n_strips = (int32_t)hm.n_strips; p.n_segs = (int32_t)hm.n_segs;
+    p.nkb = hm.nkb; p.mask_rows = hm.mask_rows; p.K_L = hm.fmt.K_L;
+    p.slot_bytes = g.slot_bytes;
+    p.x_fast = (hm.K % 32 == 0) ? 2 : (hm.K % 8 == 0) ? 1 : 0;
+    p.fp16_out = x_scale ? 1 : 0;
+    switch (g.nt) {
+        case 1: e = launch_nt<1>(p, h->sm_count, g.warps * 32, g.smem, st); break;
+        case 2: e = launch_nt<2>(p, h->sm_count, g.warps * 32, g.smem, st); break;
+        case 4: e = launch_nt<4>(p, h->sm_count, g.warps * 32, g.smem, st); break;
+        default: e = launch_nt<8>(p, h->sm_count, g.warps * 32, g.smem, st); break;
+    }
+    if (e != cudaSuccess) { h->sticky = e; return US_ERR_CUDA; }
+    return US_OK;
+}
+
 us_status us_last_error(us_handle* h)
 {
     if (!h) return US_ERR_INVALID_ARG;
@@ -411,6 +493,7 @@ const char* us_status_string(us_status s)
         case US_ERR_ALLOC: return "allocation failed";
         case US_ERR_CUDA: return "CUDA error";
         case US_ERR_DEVICE_TIMEOUT: return "bounded device wait ran out";
+        case US_ERR_SCRATCH_TOO_SMALL: return "problem needs more scratch than the fixed device array holds";
     }
     return "unknown status";
 }
