@@ -64,7 +64,10 @@ struct SpmmParams {
     uint32_t cta_begin[kMaxCtas + 1];
 };
 
-constexpr uint32_t kLutBytes = 256 * 32 * 4;
+constexpr int kLutRep = 8;   // copies of the selector table: lane l reads copy l % kLutRep. Eight copies
+                             // cost ~0.4 extra wavefronts per lookup (lanes sharing a copy collide only
+                             // when their entries fall in the same bank) and free 24 KB for more warps.
+constexpr uint32_t kLutBytes = 256 * kLutRep * 4;
 constexpr uint32_t kFill = 0x08080808u;
 constexpr uint32_t kErrTimeout = 1;
 constexpr int kNoRow = -2;        // "row ids not loaded yet" marker (-1 is a padding row)
@@ -350,7 +353,7 @@ __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, ui
             for (int i = 0; i < 4; ++i) {
                 const uint32_t cum = (i == 3) ? mw : (mw & ((1u << (8 * i + 8)) - 1u));
                 pos[ch][i + 1] = b8[ch] + 8u * (uint32_t)__popc(cum);
-                e[ch][i] = lut_a + prmt(mw, 0u, 0x4440u + i) * 128u;   // address of the table entry
+                e[ch][i] = lut_a + prmt(mw, 0u, 0x4440u + i) * (4u * kLutRep);   // address of the table entry
             }
             b8[ch] = pos[ch][4];
         }
@@ -448,7 +451,8 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
     // With a single K range the activations to stage are known before the CTA's tile range is:
     // fetch them (into registers) ahead of everything else.
     constexpr int kXPre = NT == 1 ? 8 : NT == 2 ? 4 : 0;   // 16-byte units of X a thread prefetches
-    const bool x_early = kXPre > 0 && (p.n_segs <= p.G) && p.x_fast == 2;
+    const int x_sh = 31 - __clz(p.K_L / 32);   // log2(units per (segment, token)) when a power of two
+    const bool x_early = kXPre > 0 && (p.n_segs <= p.G) && p.x_fast == 2 && (1 << x_sh) == p.K_L / 32;
     uint4 xpre[kXPre > 0 ? kXPre : 1];
     const int x_upr = p.K_L / 32, x_total = NT * 8 * p.n_segs * x_upr;
     if (x_early) {
@@ -458,8 +462,8 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
             const int u = threadIdx.x + b * blockDim.x;
             xpre[b] = make_uint4(0, 0, 0, 0);
             if (u < x_total) {
-                const int pi = u / x_upr, q = u - pi * x_upr;
-                const int sgl = pi / (NT * 8), n = pi - sgl * (NT * 8);
+                const int pi = u >> x_sh, q = u & (x_upr - 1);
+                const int sgl = pi / (NT * 8), n = pi & (NT * 8 - 1);
                 const int64_t k = (int64_t)sgl * p.K_L + 32 * q;
                 if (n < p.N && k < p.K)
                     xpre[b] = __ldg(reinterpret_cast<const uint4*>(p.X + (int64_t)n * ldx + k / 2));
@@ -546,18 +550,12 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
             }
         }
         // (built here: its arithmetic overlaps the offset loads issued just above)
-        // Selector table, replicated once per bank. Every thread computes the entries it needs (pure
-        // register arithmetic: no memory round trip in the prologue) and a warp writes one entry row.
-        for (int e0 = 0; e0 < 256; e0 += blockDim.x) {
-            const int m = e0 + threadIdx.x;
-            const uint32_t mine = m < 256 ? lut_entry(m) : 0u;
-            // thread (w, l) holds entry e0 + 32 w + l; row e0 + 32 w + r is broadcast from lane r
-    #pragma unroll 4
-            for (int r = 0; r < 32; ++r) {
-                const uint32_t v = __shfl_sync(0xffffffffu, mine, r);
-                const int e = e0 + 32 * warp + r;
-                if (e < 256) lut[e * 32 + lane] = v;
-            }
+        // Selector table, kLutRep copies. Every thread computes the entries it needs (pure register
+        // arithmetic: no memory round trip in the prologue).
+        for (int e = threadIdx.x; e < 256; e += blockDim.x) {
+            const uint32_t v = lut_entry(e);
+#pragma unroll
+            for (int r = 0; r < kLutRep; ++r) lut[e * kLutRep + r] = v;
         }
 #pragma unroll
         for (int s = 0; s <= STAGES; ++s) {
@@ -611,7 +609,7 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
     int pend_rb = -1;     // direct mode: strip whose contribution is issued but not yet signalled
     uint32_t pend_n = 0;  //              and the number of tiles in it
     const int t2 = (lane & 3) * 2;
-    const uint32_t lut_a = smem_u32(lut) + 4u * lane;
+    const uint32_t lut_a = smem_u32(lut) + 4u * (lane % kLutRep);
 
     const StoreCtx sctx{p.Y, p.w_scale, p.x_scale, p.acc, p.cnt, p.M, p.N, p.fp16_out};
     auto store_strip = [&](int rb, int (&v)[NT][4], int m_lo, int m_hi) {
@@ -669,8 +667,8 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
             for (int b = 0; b < kXPre; ++b) {
                 const int u = threadIdx.x + b * blockDim.x;
                 if (u < x_total) {
-                    const int pi = u / x_upr, q = u - pi * x_upr;
-                    const int sgl = pi / (NT * 8), n = pi - sgl * (NT * 8);
+                    const int pi = u >> x_sh, q = u & (x_upr - 1);
+                    const int sgl = pi / (NT * 8), n = pi & (NT * 8 - 1);
                     int32_t sacc = 0;
                     uint4 vlo, vhi;
                     uint2 t;
