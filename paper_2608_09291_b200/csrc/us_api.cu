@@ -47,6 +47,8 @@ int env_int(const char* name, int fallback)
 }
 int x_budget() { static int v = env_int("US_X_BUDGET_KB", 66) * 1024; return v; }          // int8 X of one K range
 int local_acc_budget() { static int v = env_int("US_LOCAL_ACC_KB", 16) * 1024; return v; }  // local strip sums
+int pdl_knob() { static int v = env_int("US_PDL", 1); return v; }          // programmatic dependent launch
+int half_sm_knob() { static int v = env_int("US_HALF_SM", 0); return v; }  // small problems: half an SM per CTA
 int max_warps() { static int v = std::min(16, std::max(2, env_int("US_MAX_WARPS", 16))); return v; }
 
 struct LaunchGeom {
@@ -75,6 +77,14 @@ bool plan_launch(const us_handle* h, int N, LaunchGeom* g)
     int warps = (limit - fixed) / (int)(kStages * g->slot_bytes);
     warps = std::min(warps, max_warps());
     if (warps < kMinWarps) return false;
+    // Small problems (a CTA sees only a few tiles per warp): take at most half an SM -- shared
+    // memory and registers -- so that the next launch's CTA can move in beside this one and run its
+    // latency-bound prologue under this one's decode (programmatic dependent launch).
+    const int64_t per_cta = (h->host.n_items + 147) / 148;
+    if (half_sm_knob() && per_cta <= 3 * (int64_t)warps) {
+        const int half = limit / 2 - 2048;
+        while (warps > 4 && (fixed + warps * kStages * (int)g->slot_bytes > half || warps > 8)) --warps;
+    }
     g->warps = warps;
     g->smem = fixed + warps * kStages * (int)g->slot_bytes;
     return true;
@@ -98,8 +108,9 @@ void plan_classes(us_handle* h, int n_cta, std::vector<uint32_t> (&sched)[4])
     }
 }
 
-int chains_knob() { static int v = env_int("US_CHAINS", 1); return v; }
 int run_knob() { static int v = env_int("US_RUN", 0); return v; }
+int chains_knob() { static int v = env_int("US_CHAINS", 1); return v; }
+
 
 // decode chains per tile: as many as the knob asks for and the tile's mask words divide into
 int chains_for(int mask_rows)
@@ -112,9 +123,21 @@ int chains_for(int mask_rows)
 template <int NT, int CH>
 cudaError_t launch_ch(const us::SpmmParams& p, int grid, int block, int smem, cudaStream_t st)
 {
-    if (p.s_local > 0) us::us_spmm_kernel<NT, kStages, CH, true><<<grid, block, smem, st>>>(p);
-    else us::us_spmm_kernel<NT, kStages, CH, false><<<grid, block, smem, st>>>(p);
-    return cudaGetLastError();
+    // Launched with programmatic stream serialization: the kernel may start while its predecessor
+    // in the stream is still running; it waits (griddepcontrol.wait) before it touches anything
+    // an earlier kernel could produce or still use.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)block);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = pdl_knob() ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (p.s_local > 0) return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, kStages, CH, true>, p);
+    return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, kStages, CH, false>, p);
 }
 
 template <int NT>

@@ -447,30 +447,10 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
         (reinterpret_cast<uintptr_t>(off_s + 2 * kOffTable) + 127) & ~uintptr_t(127));
     uint8_t* my_ring = ring0 + (size_t)warp * STAGES * p.slot_bytes;
 
-    // ---- prologue: the latency-critical small loads go out first ------------------------------
-    // With a single K range the activations to stage are known before the CTA's tile range is:
-    // fetch them (into registers) ahead of everything else.
-    constexpr int kXPre = NT == 1 ? 8 : NT == 2 ? 4 : 0;   // 16-byte units of X a thread prefetches
-    const int x_sh = 31 - __clz(p.K_L / 32);   // log2(units per (segment, token)) when a power of two
-    const bool x_early = kXPre > 0 && (p.n_segs <= p.G) && p.x_fast == 2 && (1 << x_sh) == p.K_L / 32;
-    uint4 xpre[kXPre > 0 ? kXPre : 1];
-    const int x_upr = p.K_L / 32, x_total = NT * 8 * p.n_segs * x_upr;
-    if (x_early) {
-        const int64_t ldx = ((int64_t)p.K + 1) / 2;
-#pragma unroll
-        for (int b = 0; b < kXPre; ++b) {
-            const int u = threadIdx.x + b * blockDim.x;
-            xpre[b] = make_uint4(0, 0, 0, 0);
-            if (u < x_total) {
-                const int pi = u >> x_sh, q = u & (x_upr - 1);
-                const int sgl = pi / (NT * 8), n = pi & (NT * 8 - 1);
-                const int64_t k = (int64_t)sgl * p.K_L + 32 * q;
-                if (n < p.N && k < p.K)
-                    xpre[b] = __ldg(reinterpret_cast<const uint4*>(p.X + (int64_t)n * ldx + k / 2));
-            }
-        }
-    }
     const uint32_t beg = p.cta_begin[blockIdx.x], end = p.cta_begin[blockIdx.x + 1];
+    // Programmatic dependent launch: let the next kernel of the stream start its own prologue
+    // (parameter fetch, offsets, first weight tiles) while this one is still working.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (beg >= end) return;
 #ifndef US_EXP_EPI_TIMERS
     if (timing) dbg[0] = clock64() - t_start;
@@ -604,6 +584,32 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
         }
     };
 
+    // Everything above (schedule, offsets, selector table, the first weight-tile copies) depends on
+    // nothing an earlier kernel of the stream produces. X may be the output of the kernel before,
+    // and Y / the workspace may still be in use by it: wait for the stream's earlier work here.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // With a single K range the activations to stage are known up front: fetch them into
+    // registers now, ahead of the staging pass.
+    constexpr int kXPre = NT == 1 ? 8 : NT == 2 ? 4 : 0;   // 16-byte units of X a thread prefetches
+    const int x_sh = 31 - __clz(p.K_L / 32);   // log2(units per (segment, token)) when a power of two
+    const bool x_early = kXPre > 0 && (p.n_segs <= p.G) && p.x_fast == 2 && (1 << x_sh) == p.K_L / 32;
+    uint4 xpre[kXPre > 0 ? kXPre : 1];
+    const int x_upr = p.K_L / 32, x_total = NT * 8 * p.n_segs * x_upr;
+    if (x_early) {
+        const int64_t ldx = ((int64_t)p.K + 1) / 2;
+#pragma unroll
+        for (int b = 0; b < kXPre; ++b) {
+            const int u = threadIdx.x + b * blockDim.x;
+            xpre[b] = make_uint4(0, 0, 0, 0);
+            if (u < x_total) {
+                const int pi = u >> x_sh, q = u & (x_upr - 1);
+                const int sgl = pi / (NT * 8), n = pi & (NT * 8 - 1);
+                const int64_t k = (int64_t)sgl * p.K_L + 32 * q;
+                if (n < p.N && k < p.K)
+                    xpre[b] = __ldg(reinterpret_cast<const uint4*>(p.X + (int64_t)n * ldx + k / 2));
+            }
+        }
+    }
     uint32_t phase = 0;   // bit s = parity to wait for on stage s
     bool dead = false;    // a bounded wait ran out: stop working, keep the barriers balanced
     int pend_rb = -1;     // direct mode: strip whose contribution is issued but not yet signalled
