@@ -456,7 +456,7 @@ def run_only(args):
         for k, v in binding.us_stage_timers(sw.handle, 0, read=True).items():
             tm[k] = tm.get(k, 0) + v
     per_warp = ("wait", "decode", "epilogue", "lifetime", "prologue")
-    timers = {k: (v / tm["warps"] if k in per_warp else v / len(case.sw)) for k, v in tm.items()}
+    timers = {k: (v / max(1, tm["warps"]) if k in per_warp else v / len(case.sw)) for k, v in tm.items()}
     print(json.dumps({"only": args.only, "us_per_launch_graph": t_graph * 1e6, "gbs_graph": alg / t_graph / 1e9,
                       "us_per_launch_stream_order": t * 1e6, "alg_bytes": alg,
                       "stored_bytes": binding.us_spmm_bytes(case.sw[0].handle, N, fp16),

@@ -109,19 +109,8 @@ void plan_classes(us_handle* h, int n_cta, std::vector<uint32_t> (&sched)[4])
 }
 
 int run_knob() { static int v = env_int("US_RUN", 0); return v; }
-int chains_knob() { static int v = env_int("US_CHAINS", 1); return v; }
-
-
-// decode chains per tile: as many as the knob asks for and the tile's mask words divide into
-int chains_for(int mask_rows)
-{
-    const int want = chains_knob();
-    if (want >= 2 && mask_rows % 2 == 0) return 2;
-    return 1;
-}
-
-template <int NT, int CH>
-cudaError_t launch_ch(const us::SpmmParams& p, int grid, int block, int smem, cudaStream_t st)
+template <int NT>
+cudaError_t launch_nt(const us::SpmmParams& p, int grid, int block, int smem, cudaStream_t st)
 {
     // Launched with programmatic stream serialization: the kernel may start while its predecessor
     // in the stream is still running; it waits (griddepcontrol.wait) before it touches anything
@@ -136,34 +125,23 @@ cudaError_t launch_ch(const us::SpmmParams& p, int grid, int block, int smem, cu
     attr[0].val.programmaticStreamSerializationAllowed = pdl_knob() ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (p.s_local > 0) return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, kStages, CH, true>, p);
-    return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, kStages, CH, false>, p);
-}
-
-template <int NT>
-cudaError_t launch_nt(const us::SpmmParams& p, int grid, int block, int smem, cudaStream_t st)
-{
-    switch (chains_for(p.mask_rows)) {
-        case 2: return launch_ch<NT, 2>(p, grid, block, smem, st);
-        default: return launch_ch<NT, 1>(p, grid, block, smem, st);
-    }
+    const bool la = p.s_local > 0, timed = p.timers != nullptr;
+    if (la && !timed) return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, kStages, true, false>, p);
+    if (!la && !timed) return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, kStages, false, false>, p);
+    if (la) return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, kStages, true, true>, p);
+    return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, kStages, false, true>, p);
 }
 
 // Opt every kernel variant in to the device's full dynamic shared memory (once per handle, at
 // encode time, so that us_spmm itself is nothing but a launch).
-template <int NT, int CH>
-cudaError_t enable_large_smem_ch(int bytes)
-{
-    const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
-    cudaError_t e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, kStages, CH, true>, attr, bytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, kStages, CH, false>, attr, bytes);
-    return e;
-}
 template <int NT>
 cudaError_t enable_large_smem_nt(int bytes)
 {
-    cudaError_t e = enable_large_smem_ch<NT, 1>(bytes);
-    if (e == cudaSuccess) e = enable_large_smem_ch<NT, 2>(bytes);
+    const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
+    cudaError_t e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, kStages, true, false>, attr, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, kStages, false, false>, attr, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, kStages, true, true>, attr, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, kStages, false, true>, attr, bytes);
     return e;
 }
 cudaError_t enable_large_smem(int bytes)
@@ -318,11 +296,12 @@ us_status us_spmm(us_handle* h, const void* X, int32_t N, const void* x_scale, v
         p.mg_g = magic((uint64_t)p.G);
         p.mg_glast = magic((uint64_t)g_last);
         p.mg_krs = magic((uint64_t)hm.n_strips * (uint64_t)p.G);
-        // Claim runs of up to half a strip's segments of the range (the partial sums of a run stay
-        // in registers), but never so long that a CTA's warps run out of runs to share.
+        // Claim runs of up to a whole strip's segments of the range (the partial sums of a run stay
+        // in registers; the kernel shortens the runs towards the end of a CTA's range), but never
+        // so long that a CTA's warps run out of runs to share.
         const int64_t per_cta = std::max<int64_t>(1, hm.n_items / std::max(1, h->sm_count));
         const int balanced = (int)std::max<int64_t>(1, per_cta / (4 * (int64_t)g.warps));
-        const int want = run_knob() > 0 ? run_knob() : std::min(std::max(1, p.G / 2), balanced);
+        const int want = run_knob() > 0 ? run_knob() : std::min(p.G, 2 * balanced);
         p.run_len = std::max(1, std::min(want, p.G));
     }
     p.row_order = h->d_row_order; p.w_scale = h->d_w_scale;
@@ -404,7 +383,7 @@ us_status us_spmm_static_scratch(us_handle* h, const void* X, int32_t N, const v
         p.mg_krs = magic((uint64_t)hm.n_strips * (uint64_t)p.G);
         const int64_t per_cta = std::max<int64_t>(1, hm.n_items / std::max(1, h->sm_count));
         const int balanced = (int)std::max<int64_t>(1, per_cta / (4 * (int64_t)g.warps));
-        const int want = run_knob() > 0 ? run_knob() : std::min(std::max(1, p.G / 2), balanced);
+        const int want = run_knob() > 0 ? run_knob() : std::min(p.G, 2 * balanced);
         p.run_len = std::max(1, std::min(want, p.G));
     }
     p.row_order = h->d_row_order; p.w_scale = h->d_w_scale;

@@ -423,12 +423,14 @@ __device__ __forceinline__ uint32_t fdiv(uint32_t u, unsigned long long m)
 }
 
 // LA = local mode (shared-memory strip accumulators), else direct mode.
-template <int NT, int STAGES, int CH, bool LA>
+// TIMED = record the diagnostic stage timers (a separate instantiation, so that the production
+// kernel carries none of their clock reads and branches).
+template <int NT, int STAGES, bool LA, bool TIMED>
 __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
-    const bool timing = p.timers != nullptr;
+    constexpr bool timing = TIMED;
     long long t_wait = 0, t_decode = 0, t_epi = 0, t_start = timing ? clock64() : 0, t_first = 0;
     long long dbg[4] = {0, 0, 0, 0};   // prologue checkpoints (cycles since t_start)
     const unsigned long long g_start = timing ? global_timer_ns() : 0;
@@ -492,10 +494,19 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
     auto next_pos = [&]() -> uint32_t {
         if (static_k < n_static * (int)R) return static_pos(static_k++);
         if (run_next == run_end) {
-            uint32_t b = 0;
-            if (lane == 0) b = atomicAdd(claim, R);
+            // Guided chunks: as long as every warp can still get a run of R (a whole strip's
+            // segments when R = G: its sums never leave the registers), hand out R; towards the end
+            // of the CTA's range halve the runs so that the warps finish together.
+            uint32_t b = 0, n = 0;
+            if (lane == 0) {
+                const uint32_t seen = *(volatile uint32_t*)claim;
+                const uint32_t left = seen < end ? end - seen : 0u;
+                n = R;
+                while (n > 1u && n * (uint32_t)n_warps > left) n >>= 1;
+                b = atomicAdd(claim, n);
+            }
             run_next = __shfl_sync(0xffffffffu, b, 0);
-            run_end = run_next + R;
+            run_end = run_next + __shfl_sync(0xffffffffu, n, 0);
         }
         return run_next++;
     };
@@ -654,6 +665,8 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
     tile_of(beg, kr_first, d0_, d1_);
     tile_of(end - 1, kr_last, d0_, d1_);
     int cur = 0;
+    int rb = 0, sgl = 0, m_lo = kNoRow, m_hi = kNoRow;   // strip / segment / row ids of the tile in hand
+    uint32_t last_u = 0xFFFFFFF0u;
     int y[NT][4];          // partial Y of the run in flight (fragment order)
     uint32_t y_n = 0;      // tiles summed in y
 #pragma unroll
@@ -738,18 +751,23 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
             const long long t1 = timing ? clock64() : 0;
 
             const uint32_t q = u - base;
-            const int rb = (int)fdiv(q, mg);
-            const int sgl = (int)(q - (uint32_t)rb * (uint32_t)g_kr);
-            // original rows of this strip's fragment rows g and g + 8: needed only when the strip is
-            // stored, fetched now so that the loads complete behind the decode
-            const int m_lo = __ldg(p.row_order + rb * 16 + (lane >> 2));
-            const int m_hi = __ldg(p.row_order + rb * 16 + (lane >> 2) + 8);
+            if (u == last_u + 1u && sgl + 1 < g_kr) {
+                ++sgl;                         // next segment of the same strip
+            } else {
+                rb = (int)fdiv(q, mg);
+                sgl = (int)(q - (uint32_t)rb * (uint32_t)g_kr);
+                // original rows of this strip's fragment rows g and g + 8: needed only when the
+                // strip is stored, fetched now so that the loads complete behind the decode
+                m_lo = __ldg(p.row_order + rb * 16 + (lane >> 2));
+                m_hi = __ldg(p.row_order + rb * 16 + (lane >> 2) + 8);
+            }
+            last_u = u;
             int c[NT][4];
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0;
             const uint32_t slot_a = smem_u32(my_ring + (size_t)cur * p.slot_bytes);
             const uint32_t xb_a = smem_u32(x8) + (lane >> 2) * xstride + 8 * (lane & 3) + sgl * p.K_L;
-            process_tile<NT, CH>(slot_a, lut_a, xb_a, xstride, p.mask_rows, lane, c);
+            process_tile<NT, 1>(slot_a, lut_a, xb_a, xstride, p.mask_rows, lane, c);
             __syncwarp();
             const long long t2c = timing ? clock64() : 0;
 

@@ -171,3 +171,32 @@ def test_other_stream(b):
     for o in outs:
         assert (o.cpu().numpy() == ref).all()
     sw.close()
+
+
+@pytest.mark.parametrize("M,K,N", [(1024, 4096, 16), (272, 16384, 8), (2048, 2048, 8)])
+def test_back_to_back_launches_share_a_handle(b, M, K, N):
+    """Consecutive launches may overlap their prologues (programmatic dependent launch). Calls on
+    one handle reuse its split-K workspace and counters, and a call's X may be the output of the
+    kernel just before it: results must be those of strictly serial execution."""
+    W = workloads.make_weight(M, K, 0.5, seed=M + K)
+    X1 = workloads.make_x(K, N, seed=1)
+    X2 = workloads.make_x(K, N, seed=2)
+    sw = b.SparseWeight(W, None, max_N=N)
+    try:
+        X1d = torch.from_numpy(b.pack_int4(X1)).cuda()
+        X2d = torch.from_numpy(b.pack_int4(X2)).cuda()
+        Xbuf = torch.empty_like(X1d)
+        outs = []
+        for i in range(12):
+            Xbuf.copy_(X1d if i % 2 == 0 else X2d)        # X written by the kernel right before
+            outs.append(sw.spmm(Xbuf, N).clone())
+            outs.append(sw.spmm(X2d if i % 2 == 0 else X1d, N))   # two SpMMs back to back
+        torch.cuda.synchronize()
+        sw.check()
+        ref1, ref2 = oracle.spmm_dense(W, X1), oracle.spmm_dense(W, X2)
+        for i in range(12):
+            a, c = outs[2 * i].cpu().numpy(), outs[2 * i + 1].cpu().numpy()
+            assert (a == (ref1 if i % 2 == 0 else ref2)).all(), i
+            assert (c == (ref2 if i % 2 == 0 else ref1)).all(), i
+    finally:
+        sw.close()
