@@ -33,7 +33,6 @@ struct us_handle {
 
 namespace {
 
-constexpr int kStages = 2;
 constexpr int kMinWarps = 2;
 
 int nt_for(int N) { return N <= 8 ? 1 : N <= 16 ? 2 : N <= 32 ? 4 : 8; }
@@ -47,12 +46,13 @@ int env_int(const char* name, int fallback)
 }
 int x_budget() { static int v = env_int("US_X_BUDGET_KB", 66) * 1024; return v; }          // int8 X of one K range
 int local_acc_budget() { static int v = env_int("US_LOCAL_ACC_KB", 16) * 1024; return v; }  // local strip sums
+int stages_knob() { static int v = env_int("US_STAGES", 0); return v; }     // ring slots per warp, 0 = automatic
 int pdl_knob() { static int v = env_int("US_PDL", 1); return v; }          // programmatic dependent launch
 int half_sm_knob() { static int v = env_int("US_HALF_SM", 0); return v; }  // small problems: half an SM per CTA
 int max_warps() { static int v = std::min(16, std::max(2, env_int("US_MAX_WARPS", 16))); return v; }
 
 struct LaunchGeom {
-    int nt, cls, warps, smem;
+    int nt, cls, warps, stages, smem;
     uint32_t slot_bytes;
 };
 
@@ -71,11 +71,18 @@ bool plan_launch(const us_handle* h, int N, LaunchGeom* g)
     g->cls = class_of(g->nt);
     const int G = h->G[g->cls], s_local = h->s_local[g->cls];
     g->slot_bytes = (h->host.max_item_bytes + 256u + 127u) & ~127u;
-    const int fixed = (int)us::kLutBytes + g->nt * 8 * (G * h->host.fmt.K_L + 32) + G * g->nt * 8 * 4 +
-                      32 * kStages * 8 + 32 * 4 + s_local * (g->nt * 128 + 1) * 4 + 2 * us::kOffTable * 4 + 128;
+    const int fixed_base = (int)us::kLutBytes + g->nt * 8 * (G * h->host.fmt.K_L + 32) + G * g->nt * 8 * 4 +
+                           32 * 4 + s_local * (g->nt * 128 + 1) * 4 + 2 * us::kOffTable * 4 + 128;
     const int limit = h->max_smem > 0 ? h->max_smem : 227 * 1024;
-    int warps = (limit - fixed) / (int)(kStages * g->slot_bytes);
-    warps = std::min(warps, max_warps());
+    // Ring depth: two slots per warp when that still gives (nearly) all the warps; else one slot per
+    // warp and more warps -- measured on the 70B-shaped FFN: 16 warps x 1 slot beat 9 warps x 2.
+    auto warps_for = [&](int stages) {
+        const int fixed = fixed_base + 32 * stages * 8;
+        return std::min((limit - fixed) / (int)(stages * g->slot_bytes), max_warps());
+    };
+    int stages = stages_knob() > 0 ? stages_knob() : (warps_for(1) >= warps_for(2) + 3 ? 1 : 2);
+    int warps = warps_for(stages);
+    const int fixed = fixed_base + 32 * stages * 8;
     if (warps < kMinWarps) return false;
     // Small problems (a CTA sees only a few tiles per warp): take at most half an SM -- shared
     // memory and registers -- so that the next launch's CTA can move in beside this one and run its
@@ -83,10 +90,11 @@ bool plan_launch(const us_handle* h, int N, LaunchGeom* g)
     const int64_t per_cta = (h->host.n_items + 147) / 148;
     if (half_sm_knob() && per_cta <= 3 * (int64_t)warps) {
         const int half = limit / 2 - 2048;
-        while (warps > 4 && (fixed + warps * kStages * (int)g->slot_bytes > half || warps > 8)) --warps;
+        while (warps > 4 && (fixed + warps * stages * (int)g->slot_bytes > half || warps > 8)) --warps;
     }
+    g->stages = stages;
     g->warps = warps;
-    g->smem = fixed + warps * kStages * (int)g->slot_bytes;
+    g->smem = fixed + warps * stages * (int)g->slot_bytes;
     return true;
 }
 
@@ -109,8 +117,8 @@ void plan_classes(us_handle* h, int n_cta, std::vector<uint32_t> (&sched)[4])
 }
 
 int run_knob() { static int v = env_int("US_RUN", 0); return v; }
-template <int NT>
-cudaError_t launch_nt(const us::SpmmParams& p, int grid, int block, int smem, cudaStream_t st)
+template <int NT, int ST>
+cudaError_t launch_st(const us::SpmmParams& p, int grid, int block, int smem, cudaStream_t st)
 {
     // Launched with programmatic stream serialization: the kernel may start while its predecessor
     // in the stream is still running; it waits (griddepcontrol.wait) before it touches anything
@@ -126,22 +134,35 @@ cudaError_t launch_nt(const us::SpmmParams& p, int grid, int block, int smem, cu
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     const bool la = p.s_local > 0, timed = p.timers != nullptr;
-    if (la && !timed) return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, kStages, true, false>, p);
-    if (!la && !timed) return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, kStages, false, false>, p);
-    if (la) return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, kStages, true, true>, p);
-    return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, kStages, false, true>, p);
+    if (la && !timed) return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, ST, true, false>, p);
+    if (!la && !timed) return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, ST, false, false>, p);
+    if (la) return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, ST, true, true>, p);
+    return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, ST, false, true>, p);
+}
+
+template <int NT>
+cudaError_t launch_nt(const us::SpmmParams& p, int stages, int grid, int block, int smem, cudaStream_t st)
+{
+    return stages == 1 ? launch_st<NT, 1>(p, grid, block, smem, st) : launch_st<NT, 2>(p, grid, block, smem, st);
 }
 
 // Opt every kernel variant in to the device's full dynamic shared memory (once per handle, at
 // encode time, so that us_spmm itself is nothing but a launch).
+template <int NT, int ST>
+cudaError_t enable_large_smem_st(int bytes)
+{
+    const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
+    cudaError_t e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, ST, true, false>, attr, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, ST, false, false>, attr, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, ST, true, true>, attr, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, ST, false, true>, attr, bytes);
+    return e;
+}
 template <int NT>
 cudaError_t enable_large_smem_nt(int bytes)
 {
-    const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
-    cudaError_t e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, kStages, true, false>, attr, bytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, kStages, false, false>, attr, bytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, kStages, true, true>, attr, bytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, kStages, false, true>, attr, bytes);
+    cudaError_t e = enable_large_smem_st<NT, 1>(bytes);
+    if (e == cudaSuccess) e = enable_large_smem_st<NT, 2>(bytes);
     return e;
 }
 cudaError_t enable_large_smem(int bytes)
@@ -319,10 +340,10 @@ us_status us_spmm(us_handle* h, const void* X, int32_t N, const void* x_scale, v
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e;
     switch (g.nt) {
-        case 1: e = launch_nt<1>(p, h->sm_count, g.warps * 32, g.smem, st); break;
-        case 2: e = launch_nt<2>(p, h->sm_count, g.warps * 32, g.smem, st); break;
-        case 4: e = launch_nt<4>(p, h->sm_count, g.warps * 32, g.smem, st); break;
-        default: e = launch_nt<8>(p, h->sm_count, g.warps * 32, g.smem, st); break;
+        case 1: e = launch_nt<1>(p, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
+        case 2: e = launch_nt<2>(p, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
+        case 4: e = launch_nt<4>(p, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
+        default: e = launch_nt<8>(p, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
     }
     if (e != cudaSuccess) { h->sticky = e; return US_ERR_CUDA; }
     return US_OK;
@@ -401,10 +422,10 @@ us_status us_spmm_static_scratch(us_handle* h, const void* X, int32_t N, const v
     p.x_fast = (hm.K % 32 == 0) ? 2 : (hm.K % 8 == 0) ? 1 : 0;
     p.fp16_out = x_scale ? 1 : 0;
     switch (g.nt) {
-        case 1: e = launch_nt<1>(p, h->sm_count, g.warps * 32, g.smem, st); break;
-        case 2: e = launch_nt<2>(p, h->sm_count, g.warps * 32, g.smem, st); break;
-        case 4: e = launch_nt<4>(p, h->sm_count, g.warps * 32, g.smem, st); break;
-        default: e = launch_nt<8>(p, h->sm_count, g.warps * 32, g.smem, st); break;
+        case 1: e = launch_nt<1>(p, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
+        case 2: e = launch_nt<2>(p, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
+        case 4: e = launch_nt<4>(p, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
+        default: e = launch_nt<8>(p, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
     }
     if (e != cudaSuccess) { h->sticky = e; return US_ERR_CUDA; }
     return US_OK;
