@@ -599,13 +599,17 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
     // nothing an earlier kernel of the stream produces. X may be the output of the kernel before,
     // and Y / the workspace may still be in use by it: wait for the stream's earlier work here.
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    // With a single K range the activations to stage are known up front: fetch them into
-    // registers now, ahead of the staging pass.
+    // The activations of the CTA's first K range: fetch them into registers now, ahead of the
+    // staging pass.
+    int kr_first, kr_last, d0_, d1_;
+    tile_of(beg, kr_first, d0_, d1_);
+    tile_of(end - 1, kr_last, d0_, d1_);
+    const int g_first = (kr_first == n_kr - 1) ? g_last : p.G;   // segments in that range
     constexpr int kXPre = NT == 1 ? 8 : NT == 2 ? 4 : 0;   // 16-byte units of X a thread prefetches
     const int x_sh = 31 - __clz(p.K_L / 32);   // log2(units per (segment, token)) when a power of two
-    const bool x_early = kXPre > 0 && (p.n_segs <= p.G) && p.x_fast == 2 && (1 << x_sh) == p.K_L / 32;
+    const bool x_early = kXPre > 0 && p.x_fast == 2 && (1 << x_sh) == p.K_L / 32;
     uint4 xpre[kXPre > 0 ? kXPre : 1];
-    const int x_upr = p.K_L / 32, x_total = NT * 8 * p.n_segs * x_upr;
+    const int x_upr = p.K_L / 32, x_total = NT * 8 * g_first * x_upr;
     if (x_early) {
         const int64_t ldx = ((int64_t)p.K + 1) / 2;
 #pragma unroll
@@ -615,7 +619,7 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
             if (u < x_total) {
                 const int pi = u >> x_sh, q = u & (x_upr - 1);
                 const int sgl = pi / (NT * 8), n = pi & (NT * 8 - 1);
-                const int64_t k = (int64_t)sgl * p.K_L + 32 * q;
+                const int64_t k = (int64_t)(kr_first * p.G + sgl) * p.K_L + 32 * q;
                 if (n < p.N && k < p.K)
                     xpre[b] = __ldg(reinterpret_cast<const uint4*>(p.X + (int64_t)n * ldx + k / 2));
             }
@@ -661,9 +665,6 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
         }
     };
 
-    int kr_first, kr_last, d0_, d1_;
-    tile_of(beg, kr_first, d0_, d1_);
-    tile_of(end - 1, kr_last, d0_, d1_);
     int cur = 0;
     int rb = 0, sgl = 0, m_lo = kNoRow, m_hi = kNoRow;   // strip / segment / row ids of the tile in hand
     uint32_t last_u = 0xFFFFFFF0u;
@@ -705,7 +706,7 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
                     }
                 }
             }
-            stage_x<NT>(p, 0, g_kr, x8, xstride, sx16, kXPre * (int)blockDim.x);
+            stage_x<NT>(p, kr * p.G, g_kr, x8, xstride, sx16, kXPre * (int)blockDim.x);
         } else {
             stage_x<NT>(p, kr * p.G, g_kr, x8, xstride, sx16, 0);
         }
@@ -716,7 +717,7 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
 #endif
     // The first range is staged here, outside the loop, so that the prefetched X registers are
     // dead before the decode loop starts.
-    stage_range(kr_first, (kr_first == n_kr - 1) ? g_last : p.G, x_early);
+    stage_range(kr_first, g_first, x_early);
 #ifndef US_EXP_EPI_TIMERS
     if (timing) dbg[3] = clock64() - t_start;
 #endif
