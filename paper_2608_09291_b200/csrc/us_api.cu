@@ -47,12 +47,13 @@ int env_int(const char* name, int fallback)
 int x_budget() { static int v = env_int("US_X_BUDGET_KB", 66) * 1024; return v; }          // int8 X of one K range
 int local_acc_budget() { static int v = env_int("US_LOCAL_ACC_KB", 16) * 1024; return v; }  // local strip sums
 int stages_knob() { static int v = env_int("US_STAGES", 0); return v; }     // ring slots per warp, 0 = automatic
+int lut_rep_knob() { static int v = env_int("US_LUT_REP", 0); return v; }   // selector-table copies, 0 = automatic
 int pdl_knob() { static int v = env_int("US_PDL", 1); return v; }          // programmatic dependent launch
 int half_sm_knob() { static int v = env_int("US_HALF_SM", 0); return v; }  // small problems: half an SM per CTA
 int max_warps() { static int v = std::min(16, std::max(2, env_int("US_MAX_WARPS", 16))); return v; }
 
 struct LaunchGeom {
-    int nt, cls, warps, stages, smem;
+    int nt, cls, warps, stages, smem, lut_rep;
     uint32_t slot_bytes;
 };
 
@@ -71,8 +72,13 @@ bool plan_launch(const us_handle* h, int N, LaunchGeom* g)
     g->cls = class_of(g->nt);
     const int G = h->G[g->cls], s_local = h->s_local[g->cls];
     g->slot_bytes = (h->host.max_item_bytes + 256u + 127u) & ~127u;
-    const int fixed_base = (int)us::kLutBytes + g->nt * 8 * (G * h->host.fmt.K_L + 32) + G * g->nt * 8 * 4 +
+    // selector table copies: 32 (conflict-free lookups) when that costs no warp, else 8
+    int lut_rep = 32;
+    auto fixed_for = [&](int rep) {
+        return 256 * rep * 4 + (int)us::kLutScratchBytes + g->nt * 8 * (G * h->host.fmt.K_L + 32) + G * g->nt * 8 * 4 +
                            32 * 4 + s_local * (g->nt * 128 + 1) * 4 + 2 * us::kOffTable * 4 + 128;
+    };
+    int fixed_base = fixed_for(lut_rep);
     const int limit = h->max_smem > 0 ? h->max_smem : 227 * 1024;
     // Ring depth: two slots per warp when that still gives (nearly) all the warps; else one slot per
     // warp and more warps -- measured on the 70B-shaped FFN: 16 warps x 1 slot beat 9 warps x 2.
@@ -80,6 +86,16 @@ bool plan_launch(const us_handle* h, int N, LaunchGeom* g)
         const int fixed = fixed_base + 32 * stages * 8;
         return std::min((limit - fixed) / (int)(stages * g->slot_bytes), max_warps());
     };
+    {
+        const int w32 = std::max(warps_for(1), warps_for(2));
+        fixed_base = fixed_for(8);
+        const int w8 = std::max(warps_for(1), warps_for(2));
+        // 32 copies only for long-running CTAs (measured: 1 % faster on the 70B-shaped FFN, but the
+        // 4096 x 4096 case -- about one tile per warp -- loses 5 % to the bigger table)
+        const bool long_run = (h->host.n_items + 147) / 148 >= 4 * (int64_t)w8;
+        if (w32 >= w8 && long_run) { lut_rep = 32; fixed_base = fixed_for(32); } else { lut_rep = 8; }
+        if (lut_rep_knob() == 8 || lut_rep_knob() == 32) { lut_rep = lut_rep_knob(); fixed_base = fixed_for(lut_rep); }
+    }
     int stages = stages_knob() > 0 ? stages_knob() : (warps_for(1) >= warps_for(2) + 3 ? 1 : 2);
     int warps = warps_for(stages);
     const int fixed = fixed_base + 32 * stages * 8;
@@ -93,6 +109,7 @@ bool plan_launch(const us_handle* h, int N, LaunchGeom* g)
         while (warps > 4 && (fixed + warps * stages * (int)g->slot_bytes > half || warps > 8)) --warps;
     }
     g->stages = stages;
+    g->lut_rep = lut_rep;
     g->warps = warps;
     g->smem = fixed + warps * stages * (int)g->slot_bytes;
     return true;
@@ -309,7 +326,7 @@ us_status us_spmm(us_handle* h, const void* X, int32_t N, const void* x_scale, v
     us::SpmmParams p;
     p.blob = h->d_blob; p.item_off = h->d_item_off;
     std::memcpy(p.cta_begin, h->cta_begin[g.cls].data(), h->cta_begin[g.cls].size() * sizeof(uint32_t));
-    p.G = h->G[g.cls]; p.s_local = h->s_local[g.cls];
+    p.G = h->G[g.cls]; p.s_local = h->s_local[g.cls]; p.lut_rep = g.lut_rep;
     {
         const int64_t n_kr = (hm.n_segs + p.G - 1) / p.G;
         const int64_t g_last = hm.n_segs - (n_kr - 1) * p.G;
@@ -394,7 +411,7 @@ us_status us_spmm_static_scratch(us_handle* h, const void* X, int32_t N, const v
     us::SpmmParams p;
     p.blob = h->d_blob; p.item_off = h->d_item_off;
     std::memcpy(p.cta_begin, h->cta_begin[g.cls].data(), h->cta_begin[g.cls].size() * sizeof(uint32_t));
-    p.G = h->G[g.cls]; p.s_local = h->s_local[g.cls];
+    p.G = h->G[g.cls]; p.s_local = h->s_local[g.cls]; p.lut_rep = g.lut_rep;
     {
         const int64_t n_kr = (hm.n_segs + p.G - 1) / p.G;
         const int64_t g_last = hm.n_segs - (n_kr - 1) * p.G;

@@ -55,6 +55,7 @@ struct SpmmParams {
     unsigned long long mg_g, mg_glast, mg_krs;  // floor(2^40/d)+1 for d = G, the last range's
                                                 // segment count, n_strips * G
     int32_t s_local;            // local mode: strips a CTA may hold in shared memory (0 = direct mode)
+    int32_t lut_rep;            // copies of the selector table in shared memory (8 or 32)
     int32_t nkb, mask_rows, K_L;
     uint32_t slot_bytes;        // ring slot size (max tile blob + slack), multiple of 128
     int32_t x_fast;             // 2: K % 32 == 0 (16-byte loads); 1: K % 8 == 0 (4-byte loads); 0: bytes
@@ -64,14 +65,14 @@ struct SpmmParams {
     uint32_t cta_begin[kMaxCtas + 1];
 };
 
-constexpr int kLutRep = 8;   // copies of the selector table: lane l reads copy l % kLutRep. Eight copies
+constexpr int kLutRepMax = 32;   // copies of the selector table: lane l reads copy l % kLutRep. Eight copies
                              // cost ~0.4 extra wavefronts per lookup (lanes sharing a copy collide only
                              // when their entries fall in the same bank) and free 24 KB for more warps.
-constexpr uint32_t kLutBytes = 256 * kLutRep * 4;
+constexpr uint32_t kLutScratchBytes = 256 * 4;   // one unreplicated copy, built first
 constexpr uint32_t kFill = 0x08080808u;
 constexpr uint32_t kErrTimeout = 1;
 constexpr int kNoRow = -2;        // "row ids not loaded yet" marker (-1 is a padding row)
-constexpr int kOffTable = 384;   // tile offsets of a CTA kept in shared memory (start, end pairs)
+constexpr int kOffTable = 256;   // tile offsets of a CTA kept in shared memory (start, end pairs)
 
 // ---- selector table -------------------------------------------------------------------------
 // entry(m): low 16 bits  = prmt selector for mask bits 0..3 reading the 4 bytes AT the lane's
@@ -320,8 +321,9 @@ __device__ __forceinline__ void store_rows(const StoreCtx p, const int (&v)[NT][
 // All addresses are 32-bit shared-memory addresses: slot_a = the staged tile, lut_a = selector
 // table + 4*lane, xb_a = this lane's first B-fragment of the tile's segment.
 template <int NT, int CH>
-__device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, uint32_t xb_a,
-                                             int xstride, int mask_rows, int lane, int (&c)[NT][4])
+__device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, uint32_t lut_stride,
+                                             uint32_t xb_a, int xstride, int mask_rows, int lane,
+                                             int (&c)[NT][4])
 {
     const int rows_per = mask_rows / CH;
     const uint32_t mask_a = slot_a + 4u * lane;
@@ -353,7 +355,7 @@ __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, ui
             for (int i = 0; i < 4; ++i) {
                 const uint32_t cum = (i == 3) ? mw : (mw & ((1u << (8 * i + 8)) - 1u));
                 pos[ch][i + 1] = b8[ch] + 8u * (uint32_t)__popc(cum);
-                e[ch][i] = lut_a + prmt(mw, 0u, 0x4440u + i) * (4u * kLutRep);   // address of the table entry
+                e[ch][i] = lut_a + prmt(mw, 0u, 0x4440u + i) * lut_stride;   // address of the table entry
             }
             b8[ch] = pos[ch][4];
         }
@@ -437,8 +439,9 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
 
     // ---- shared-memory carve-up (mirrored by plan_launch on the host) --------------------------
     const int xstride = p.G * p.K_L + 32;
-    uint32_t* lut = reinterpret_cast<uint32_t*>(smem);
-    uint8_t* x8 = smem + kLutBytes;
+    uint32_t* lut = reinterpret_cast<uint32_t*>(smem);                       // [256][lut_rep]
+    uint32_t* lut1 = lut + 256 * p.lut_rep;                                  // [256] built first
+    uint8_t* x8 = reinterpret_cast<uint8_t*>(lut1 + 256);
     int32_t* sx16 = reinterpret_cast<int32_t*>(x8 + NT * 8 * xstride);
     uint64_t* bars = reinterpret_cast<uint64_t*>(sx16 + p.G * NT * 8);
     uint32_t* claim = reinterpret_cast<uint32_t*>(bars + 32 * STAGES);
@@ -541,13 +544,9 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
             }
         }
         // (built here: its arithmetic overlaps the offset loads issued just above)
-        // Selector table, kLutRep copies. Every thread computes the entries it needs (pure register
-        // arithmetic: no memory round trip in the prologue).
-        for (int e = threadIdx.x; e < 256; e += blockDim.x) {
-            const uint32_t v = lut_entry(e);
-#pragma unroll
-            for (int r = 0; r < kLutRep; ++r) lut[e * kLutRep + r] = v;
-        }
+        // Selector table: every thread computes one entry (pure register arithmetic: no memory
+        // round trip in the prologue); the copies are written after the next CTA barrier.
+        for (int e = threadIdx.x; e < 256; e += blockDim.x) lut1[e] = lut_entry(e);
 #pragma unroll
         for (int s = 0; s <= STAGES; ++s) {
             const uint32_t a = __shfl_sync(0xffffffffu, o0, s), b = __shfl_sync(0xffffffffu, o1, s);
@@ -630,7 +629,7 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
     int pend_rb = -1;     // direct mode: strip whose contribution is issued but not yet signalled
     uint32_t pend_n = 0;  //              and the number of tiles in it
     const int t2 = (lane & 3) * 2;
-    const uint32_t lut_a = smem_u32(lut) + 4u * (lane % kLutRep);
+    const uint32_t lut_a = smem_u32(lut) + 4u * (uint32_t)(lane & (p.lut_rep - 1));
 
     const StoreCtx sctx{p.Y, p.w_scale, p.x_scale, p.acc, p.cnt, p.M, p.N, p.fp16_out};
     auto store_strip = [&](int rb, int (&v)[NT][4], int m_lo, int m_hi) {
@@ -681,6 +680,8 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
             for (int i = threadIdx.x; i < p.s_local; i += blockDim.x) cnt_l[i] = 0;
         }
         __syncthreads();
+        // copies of the selector table: entry e, copy r at word e * lut_rep + r (conflict-free writes)
+        for (int i = threadIdx.x, sh = 31 - __clz(p.lut_rep); i < 256 * p.lut_rep; i += blockDim.x) lut[i] = lut1[i >> sh];
         if (use_prefetched) {
             // expand the prefetched units; anything beyond them goes through the general path
 #pragma unroll
@@ -768,7 +769,7 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
             for (int nt = 0; nt < NT; ++nt) c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0;
             const uint32_t slot_a = smem_u32(my_ring + (size_t)cur * p.slot_bytes);
             const uint32_t xb_a = smem_u32(x8) + (lane >> 2) * xstride + 8 * (lane & 3) + sgl * p.K_L;
-            process_tile<NT, 1>(slot_a, lut_a, xb_a, xstride, p.mask_rows, lane, c);
+            process_tile<NT, 1>(slot_a, lut_a, 4u * (uint32_t)p.lut_rep, xb_a, xstride, p.mask_rows, lane, c);
             __syncwarp();
             const long long t2c = timing ? clock64() : 0;
 
