@@ -45,7 +45,7 @@ int env_int(const char* name, int fallback)
     return (v && *v) ? std::atoi(v) : fallback;
 }
 int x_budget() { static int v = env_int("US_X_BUDGET_KB", 66) * 1024; return v; }          // int8 X of one K range
-int local_acc_budget() { static int v = env_int("US_LOCAL_ACC_KB", 16) * 1024; return v; }  // local strip sums
+int local_acc_budget() { static int v = env_int("US_LOCAL_ACC_KB", 32) * 1024; return v; }  // local strip sums
 int stages_knob() { static int v = env_int("US_STAGES", 0); return v; }     // ring slots per warp, 0 = automatic
 int lut_rep_knob() { static int v = env_int("US_LUT_REP", 0); return v; }   // selector-table copies, 0 = automatic
 int pdl_knob() { static int v = env_int("US_PDL", 1); return v; }          // programmatic dependent launch
