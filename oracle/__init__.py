@@ -143,6 +143,21 @@ def lspd_idx_base(mask: np.ndarray, r: int, g: int, G: int) -> int:
     return int(_load().orc_lspd_idx_base(_p(mask), int(mask.shape[1]), int(r), int(g), int(G)))
 
 
+def reorder_tile(mask: np.ndarray, R_A: int, C_A: int):
+    """Alg. 1 on one local tile. mask: (H_L, K_L) array, nonzero = surviving weight.
+    Returns (perm, cost): perm[p * (H_L // R_A) + g] = the p-th row of the g-th group; cost = the
+    least number of active union-mask entries (Eq. 5 at the full row set)."""
+    lib = _load()
+    m = np.ascontiguousarray(mask != 0, dtype=np.uint8)
+    H_L, K_L = m.shape
+    perm = np.full(H_L, -1, dtype=np.int32)
+    lib.orc_reorder_tile.restype = ctypes.c_int64
+    cost = lib.orc_reorder_tile(_p(m), int(H_L), int(K_L), int(R_A), int(C_A), _p(perm))
+    if cost < 0:
+        raise ValueError("unusable reordering parameters")
+    return perm, int(cost)
+
+
 def dequant(acc: np.ndarray, s_w: np.ndarray, s_x: np.ndarray) -> np.ndarray:
     """fp16(acc[n, m] * s_w[m] * s_x[n]); the scales are fp16 inputs, the product is taken in
     float64 and rounded once to nearest-even fp16."""

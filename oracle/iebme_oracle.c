@@ -9,7 +9,8 @@
  *   - the result the SpMM kernel (paper Alg. 2: "W in IE-BME format, dense X -> Y") must
  *     reach: Y = W * X with INT32 accumulation, computed (a) as a naive triple loop on
  *     the masked dense weight and (b) straight from the encoded arrays,
- *   - the LSPD index rule (paper Sec. VI-B: idx_base + seg_rank).
+ *   - the LSPD index rule (paper Sec. VI-B: idx_base + seg_rank),
+ *   - bitmap-aware row reordering of one local tile (paper Sec. V-B, Alg. 1).
  *
  * Only tests, the smoke check and the bench's cpu-baseline leg may call this file.
  * It shares no code, header, table or constant with the CUDA library.
@@ -256,4 +257,103 @@ int orc_num_threads(void)
     }
 #endif
     return n;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Bitmap-aware row reordering (paper Sec. V-B, Eqs. 3-5, Alg. 1), one local tile at a time.
+ *
+ *   mask   : H_L x K_L bytes, nonzero = the weight at that position survives pruning
+ *   group  : R_A rows sharing one union-mask row; its cost (Eqs. 3-4) = number of grouped
+ *            columns j in [0, K_L/C_A) at which any of its rows has a nonzero in any of the
+ *            C_A column partitions (column j + c*K_L/C_A)
+ *   F(S)   : least total cost of splitting the row set S into groups (Eq. 5); memoised
+ *            recursion on the subset bitmask, always grouping the lowest row of S first
+ *   result : groups with rows ascending, groups in lexicographic order, permutation =
+ *            partition-wise concatenation: perm[p*(H_L/R_A) + g] = p-th row of group g.
+ *
+ * Ties between groupings of equal cost go to the first candidate met when the partners of the
+ * lowest row are enumerated in ascending combination order (the paper fixes no tie rule).
+ * Returns the optimal cost F(all rows), or -1 on unusable arguments (H_L > 20, R_A not
+ * dividing H_L, C_A not dividing K_L).
+ * ------------------------------------------------------------------------------------------ */
+typedef struct {
+    const uint8_t *mask;
+    int H_L, K_L, R_A, C_A;
+    int64_t *F;        /* 2^H_L entries, -1 = not computed yet */
+    uint32_t *choice;  /* the group (as a row bitmask) taken first at state S */
+} reorder_ctx;
+
+static int64_t group_cost(const reorder_ctx *c, uint32_t rows)
+{
+    const int K_B = c->K_L / c->C_A;
+    int64_t cost = 0;
+    for (int j = 0; j < K_B; ++j) {
+        int active = 0;
+        for (int r = 0; r < c->H_L && !active; ++r) {
+            if (!((rows >> r) & 1u)) continue;
+            for (int cc = 0; cc < c->C_A && !active; ++cc)
+                if (c->mask[(int64_t)r * c->K_L + j + cc * K_B]) active = 1;
+        }
+        cost += active;
+    }
+    return cost;
+}
+
+static int64_t reorder_F(reorder_ctx *c, uint32_t S);
+
+/* Extends `group` (already holding `have` rows, the last one `last`) by rows of S above
+ * `last`; at R_A rows evaluates cost + F(rest) and keeps the best. */
+static void reorder_try(reorder_ctx *c, uint32_t S, uint32_t group, int have, int last,
+                        int64_t *best, uint32_t *best_group)
+{
+    if (have == c->R_A) {
+        const int64_t v = group_cost(c, group) + reorder_F(c, S & ~group);
+        if (*best < 0 || v < *best) { *best = v; *best_group = group; }
+        return;
+    }
+    for (int r = last + 1; r < c->H_L; ++r)
+        if ((S >> r) & 1u) reorder_try(c, S, group | (1u << r), have + 1, r, best, best_group);
+}
+
+static int64_t reorder_F(reorder_ctx *c, uint32_t S)
+{
+    if (S == 0) return 0;
+    if (c->F[S] >= 0) return c->F[S];
+    int r = 0;
+    while (!((S >> r) & 1u)) ++r;
+    int64_t best = -1;
+    uint32_t best_group = 0;
+    reorder_try(c, S, 1u << r, 1, r, &best, &best_group);
+    c->F[S] = best;
+    c->choice[S] = best_group;
+    return best;
+}
+
+int64_t orc_reorder_tile(const uint8_t *mask, int H_L, int K_L, int R_A, int C_A, int32_t *perm_out)
+{
+    if (H_L <= 0 || H_L > 20 || R_A <= 0 || C_A <= 0 || H_L % R_A || K_L <= 0 || K_L % C_A) return -1;
+    reorder_ctx c = {mask, H_L, K_L, R_A, C_A, NULL, NULL};
+    const size_t n_states = (size_t)1 << H_L;
+    c.F = (int64_t *)malloc(n_states * sizeof(int64_t));
+    c.choice = (uint32_t *)calloc(n_states, sizeof(uint32_t));
+    if (!c.F || !c.choice) { free(c.F); free(c.choice); return -1; }
+    for (size_t i = 0; i < n_states; ++i) c.F[i] = -1;
+    const uint32_t all = (uint32_t)(n_states - 1);
+    const int64_t total = reorder_F(&c, all);
+
+    /* Walk the choices. Each step takes the group holding the lowest remaining row, so the
+     * groups come out ordered by their first rows -- which, rows inside a group being ascending
+     * and groups disjoint, is the lexicographic order the paper asks for. */
+    const int n_groups = H_L / R_A;
+    uint32_t S = all;
+    for (int g = 0; g < n_groups; ++g) {
+        const uint32_t grp = c.choice[S];
+        int p = 0;
+        for (int r = 0; r < H_L; ++r)
+            if ((grp >> r) & 1u) perm_out[p++ * n_groups + g] = r;
+        S &= ~grp;
+    }
+    free(c.F);
+    free(c.choice);
+    return total;
 }
