@@ -394,7 +394,76 @@ def sweep(binding, torch, workloads, l2, peak_gbs):
     run_case("attn7b_qkv_fused", 12288, 4096, 0.5, 210, [8], True)   # Q, K, V stacked: one launch
     run_case("ffn7b_up", 11008, 4096, 0.5, 300, [8], True, row_varying=True, flags=binding.US_ENCODE_SORT_ROWS)
     run_case("ffn70b_up", 28672, 8192, 0.6, 500, [1, 4, 8, 16, 32, 64], False)
+    # Bitmap-aware row pairing inside each strip (the per-strip form of Alg. 1): fewer union bits.
+    run_case("attn7b_paired", 4096, 4096, 0.5, 201, [8], True, flags=binding.US_ENCODE_PAIR_ROWS)
+    run_case("ffn70b_up_paired", 28672, 8192, 0.6, 500, [8], False, flags=binding.US_ENCODE_PAIR_ROWS)
+    for s in (0.3, 0.5, 0.7):
+        rows.append(layer_chain(binding, torch, workloads, l2, s))
     return rows
+
+
+def layer_chain(binding, torch, workloads, l2, sparsity=0.5):
+    """All seven projections of one LLaMA-2-13B-shaped decoder layer (Q, K, V, O 5120x5120; gate, up
+    13824x5120; down 5120x13824) at the given sparsity, N = 16, fp16 output, back to back on one stream
+    (one CUDA graph; consecutive launches overlap through programmatic dependent launch). Several
+    copies of the layer rotate so that the weights come from HBM."""
+    shapes = [(5120, 5120)] * 4 + [(13824, 5120)] * 2 + [(5120, 13824)]
+    N = 16
+    mats = []
+    for i, (m, k) in enumerate(shapes):
+        W = workloads.make_weight(m, k, sparsity, 410 + i)
+        s_w, _ = workloads.make_scales(m, N, 410 + i)
+        mats.append((W, s_w))
+    layer_bytes = 0
+    copies = []
+    while layer_bytes * len(copies) < 3.2 * l2 or len(copies) < 2:
+        layer = [binding.SparseWeight(W, s_w, max_N=N) for W, s_w in mats]
+        layer_bytes = sum(sw.stats["bytes_total"] for sw in layer)
+        copies.append(layer)
+    alg = sum(algorithmic_bytes(sw.stats, N, True) for sw in copies[0])
+    xs = {k: torch.from_numpy(binding.pack_int4(workloads.make_x(k, N, 77))).cuda() for k in (5120, 13824)}
+    _, s_x = workloads.make_scales(8, N, 77)
+    sxd = torch.from_numpy(s_x.copy()).cuda()
+    outs = {m: torch.empty((N, m), dtype=torch.float16, device="cuda") for m in (5120, 13824)}
+
+    def enqueue():
+        for layer in copies:
+            for sw in layer:
+                sw.spmm(xs[sw.K], N, sxd, out=outs[sw.M])
+
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        enqueue()
+    torch.cuda.current_stream().wait_stream(s)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        enqueue()
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 20
+    e0.record()
+    for _ in range(reps):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    for layer in copies:
+        for sw in layer:
+            sw.check()
+    t = e0.elapsed_time(e1) * 1e-3 / (reps * len(copies))
+    row = {"case": "layer13b_chain", "M": 0, "K": 0, "sparsity": sparsity, "N": N, "out": "fp16", "us": t * 1e6,
+           "alg_bytes": alg, "stored_bytes": layer_bytes, "gbs": alg / t / 1e9,
+           "pct_of_8tbs": 100 * alg / t / 1e9 / CONTRACT_PEAK_GBS, "frac_of_measured": alg / t / 1e9 / measured_peaks()[0],
+           "dense_equiv_tops": 2.0 * sum(m * k for m, k in shapes) * N / t / 1e12, "replicas": len(copies),
+           "pmr": copies[0][0].stats["pmr"], "launches_per_unit": len(shapes)}
+    for layer in copies:
+        for sw in layer:
+            sw.close()
+    torch.cuda.empty_cache()
+    return row
 
 
 def cpu_baseline(W, X, s_w, s_x, stats):

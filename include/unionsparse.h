@@ -68,6 +68,14 @@ typedef struct us_handle us_handle;
                                   so that rows of similar density share a strip; the output
                                   row order of us_spmm is unchanged (folded into the store)  */
 
+#define US_ENCODE_PAIR_ROWS 4u /* bitmap-aware row reordering (paper Sec. V-B, Alg. 1) in its
+                                  per-strip form: inside every 16-row strip (after SORT_ROWS, if
+                                  also given) choose which two rows share each union-mask row so
+                                  that the strip's union mask has the fewest active bits over all
+                                  of K; exact (subset DP, Eq. 5). One grouping per strip rather
+                                  than per tile, so the output row order of us_spmm is unchanged
+                                  (folded into the store) at no run-time cost                */
+
 /*
  * Offline encoder (paper Sec. V-A, Fig. 7: dense pruned INT4 -> union bitmaps, per-tile
  * offsets, packed INT4 values), followed by the upload to the current CUDA device.

@@ -20,6 +20,7 @@ _lib = ctypes.CDLL(str(_LIB_PATH))
 US_OK = 0
 US_ENCODE_HOST_ONLY = 1
 US_ENCODE_SORT_ROWS = 2
+US_ENCODE_PAIR_ROWS = 4
 
 EXPORTS = ["us_encode", "us_get_stats", "us_decode", "us_get_row_order", "us_spmm", "us_spmm_static_scratch",
            "us_last_error", "us_stage_timers", "us_destroy", "us_spmm_bytes", "us_launch_info", "us_status_string"]

@@ -44,7 +44,7 @@ int env_int(const char* name, int fallback)
     const char* v = std::getenv(name);
     return (v && *v) ? std::atoi(v) : fallback;
 }
-int x_budget() { static int v = env_int("US_X_BUDGET_KB", 66) * 1024; return v; }          // int8 X of one K range
+int x_budget() { static int v = env_int("US_X_BUDGET_KB", 0) * 1024; return v; }           // int8 X of one K range; 0 = automatic
 int local_acc_budget() { static int v = env_int("US_LOCAL_ACC_KB", 32) * 1024; return v; }  // local strip sums
 int stages_knob() { static int v = env_int("US_STAGES", 0); return v; }     // ring slots per warp, 0 = automatic
 int lut_rep_knob() { static int v = env_int("US_LUT_REP", 0); return v; }   // selector-table copies, 0 = automatic
@@ -57,11 +57,30 @@ struct LaunchGeom {
     uint32_t slot_bytes;
 };
 
-// Segments per K range for an N class: as many as keep the int8 activations within kXBudget.
-int segs_per_range(const us::HostMatrix& hm, int nt)
+// Segments per K range for an N class. The int8 activations of one K range live in shared memory
+// next to the warps' tile slots, so fewer, longer ranges (fewer partial-sum flushes) cost warps.
+// Returns the range length of the split into the fewest equal ranges, not fewer than min_ranges,
+// that still leaves room for min_warps one-slot warps (measured: 15 warps and one range beat
+// 16 warps and two ranges by 25 % on a 13824 x 5120 matrix at N = 16).
+bool plan_debug() { static int v = env_int("US_PLAN_DEBUG", 0); return v != 0; }
+int min_warps_knob() { static int v = env_int("US_MIN_WARPS", 12); return v; }
+int segs_per_range(const us::HostMatrix& hm, int nt, int limit, int64_t min_ranges)
 {
-    int g = (x_budget() / (nt * 8) - 32) / hm.fmt.K_L;
-    return (int)std::max<int64_t>(1, std::min<int64_t>(g, hm.n_segs));
+    const int64_t n_segs = hm.n_segs;
+    if (x_budget() > 0) {
+        const int g = (x_budget() / (nt * 8) - 32) / hm.fmt.K_L;
+        return (int)std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(g, n_segs), (n_segs + min_ranges - 1) / min_ranges));
+    }
+    const int slot = (int)((hm.max_item_bytes + 256u + 127u) & ~127u);
+    const int acc = nt * 512 * 2 <= local_acc_budget() ? local_acc_budget() : 0;
+    const int other = 256 * 8 * 4 + (int)us::kLutScratchBytes + acc + 2 * us::kOffTable * 4 + 1024;
+    const int want = std::min(max_warps(), min_warps_knob());
+    for (int64_t r = std::max<int64_t>(1, min_ranges); r <= n_segs; ++r) {
+        const int64_t G = (n_segs + r - 1) / r;
+        const int64_t xb = (int64_t)nt * 8 * (G * hm.fmt.K_L + 32) + G * nt * 32;
+        if ((limit - other - xb) / slot >= want) return (int)G;
+    }
+    return 1;
 }
 
 // Shared-memory layout of us_spmm_kernel: selector table, int8 X of one K range, per-(segment,
@@ -118,18 +137,31 @@ bool plan_launch(const us_handle* h, int N, LaunchGeom* g)
 // Chooses, per N class, the K-range width and whether strips are summed in shared memory.
 void plan_classes(us_handle* h, int n_cta, std::vector<uint32_t> (&sched)[4])
 {
+    const int limit = h->max_smem > 0 ? h->max_smem : 227 * 1024;
     for (int c = 0; c < 4; ++c) {
         const int nt = 1 << c;
-        int G = segs_per_range(h->host, nt), worst = 1;
-        us::make_schedule(h->host, n_cta, G, &sched[c], &worst);
-        if (G > 1 && worst * nt * 512 <= local_acc_budget()) {
-            h->G[c] = G;
-            h->s_local[c] = worst;
-        } else {  // direct mode: one segment per range, every tile goes to the global workspace
-            h->G[c] = 1;
-            h->s_local[c] = 0;
-            if (G != 1) us::make_schedule(h->host, n_cta, 1, &sched[c], &worst);
+        // Local mode needs the strip sums of a CTA's share of one K range in shared memory; a short
+        // last range spreads a CTA over more strips, so shorter ranges are tried before giving up.
+        h->G[c] = 1;
+        h->s_local[c] = 0;
+        int G = 0, worst = 1;
+        for (int64_t r = 1; r <= h->host.n_segs; ++r) {
+            const int Gr = segs_per_range(h->host, nt, limit, r);
+            if (Gr == G) continue;
+            G = Gr;
+            if (G <= 1) break;
+            us::make_schedule(h->host, n_cta, G, &sched[c], &worst);
+            if (plan_debug())
+                fprintf(stderr, "[unionsparse] plan nt=%d: G=%d needs %d local strips\n", nt, G, worst);
+            if (worst * nt * 512 <= local_acc_budget()) {
+                h->G[c] = G;
+                h->s_local[c] = worst;
+                break;
+            }
         }
+        // direct mode: one segment per range, every tile goes to the global workspace (longer ranges
+        // and runs were measured: no gain at N = 32, the bigger X costs more than the adds it saves)
+        if (h->s_local[c] == 0) us::make_schedule(h->host, n_cta, 1, &sched[c], &worst);
     }
 }
 

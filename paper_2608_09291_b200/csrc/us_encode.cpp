@@ -1,6 +1,7 @@
 // Host encoder / decoder of the lane-stream IE-BME layout (see us_host.h), statistics
 // (paper Sec. V-A storage arrays, Eq. 1) and the CTA schedule. Pure C++: no CUDA here.
 #include <algorithm>
+#include <climits>
 #include <atomic>
 #include <cstring>
 #include <numeric>
@@ -39,6 +40,65 @@ void parallel_for(int64_t n, int threads, F&& f)
             }
         });
     for (auto& th : pool) th.join();
+}
+
+// Bitmap-aware row reordering (paper Sec. V-B, Alg. 1) in its per-strip form: within each strip
+// of 16 rows, choose which rows share a union-mask row (strip rows g and g+8) so that the strip
+// activates the fewest union-mask bits over the whole K extent. One choice per strip -- not per
+// tile -- keeps every tile of a strip on the same output rows, so the kernel's store undoes it
+// through row_order at no cost. Pair costs come from 64-bit row bitsets; the least-cost perfect
+// matching is found bottom-up over all 2^16 row subsets (Eq. 5).
+void pair_rows(const int8_t* W, int64_t M, int64_t K, int threads, HostMatrix* hp)
+{
+    HostMatrix& h = *hp;
+    (void)M;
+    const int64_t words = (K + 63) / 64;
+    parallel_for(h.n_strips, threads, [&](int64_t rb, int) {
+        std::vector<uint64_t> bits((size_t)16 * words, 0);
+        for (int r = 0; r < 16; ++r) {
+            const int32_t o = h.row_order[rb * 16 + r];
+            if (o < 0) continue;
+            const int8_t* p = W + (int64_t)o * K;
+            uint64_t* b = bits.data() + (size_t)r * words;
+            for (int64_t k = 0; k < K; ++k)
+                if (p[k]) b[k >> 6] |= 1ull << (k & 63);
+        }
+        int32_t cost[16][16];
+        for (int a = 0; a < 16; ++a)
+            for (int b = a + 1; b < 16; ++b) {
+                int64_t c = 0;
+                const uint64_t *pa = bits.data() + (size_t)a * words, *pb = bits.data() + (size_t)b * words;
+                for (int64_t w = 0; w < words; ++w) c += __builtin_popcountll(pa[w] | pb[w]);
+                cost[a][b] = cost[b][a] = (int32_t)c;
+            }
+        // F[S] = least cost of pairing up the rows in S (|S| even); partner[S] = the row paired
+        // with the lowest row of S in that optimum.
+        std::vector<int32_t> F((size_t)1 << 16, 0);
+        std::vector<int8_t> partner((size_t)1 << 16, -1);
+        for (uint32_t S = 1; S < (1u << 16); ++S) {
+            if (__builtin_popcount(S) & 1) continue;
+            const int lo = __builtin_ctz(S);
+            const uint32_t rest = S & (S - 1);
+            int32_t best = INT32_MAX;
+            int8_t arg = -1;
+            for (uint32_t m = rest; m; m &= m - 1) {
+                const int b = __builtin_ctz(m);
+                const int32_t v = cost[lo][b] + F[rest & ~(1u << b)];
+                if (v < best) { best = v; arg = (int8_t)b; }
+            }
+            F[S] = best;
+            partner[S] = arg;
+        }
+        // Pairs come out ordered by their lower rows: the canonical order of the paper.
+        int32_t old_order[16], g = 0;
+        std::copy(h.row_order.begin() + rb * 16, h.row_order.begin() + rb * 16 + 16, old_order);
+        for (uint32_t S = 0xFFFFu; S; ++g) {
+            const int lo = __builtin_ctz(S), b = partner[S];
+            h.row_order[rb * 16 + g] = old_order[lo];
+            h.row_order[rb * 16 + g + 8] = old_order[b];
+            S &= ~((1u << lo) | (1u << b));
+        }
+    });
 }
 
 }  // namespace
@@ -94,6 +154,8 @@ us_status encode_host(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_s
     } else {
         std::iota(h.row_order.begin(), h.row_order.begin() + M, 0);
     }
+
+    if (flags & US_ENCODE_PAIR_ROWS) pair_rows(W, M, K, threads, &h);
 
     // ---- build every tile blob (parallel over strips) ------------------------------------
     const int K_L = fmt.K_L, nkb = h.nkb, mask_rows = h.mask_rows;

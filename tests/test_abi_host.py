@@ -31,9 +31,9 @@ def test_library_exports_every_declared_symbol(b):
 
 @pytest.mark.parametrize("M,K,s,K_L", [(64, 1024, 0.5, 1024), (37, 300, 0.5, 128), (160, 2176, 0.7, 256),
                                        (16, 128, 0.0, 128), (48, 512, 1.0, 512), (1024, 1024, 0.3, 256)])
-@pytest.mark.parametrize("flags", [0, 2])
+@pytest.mark.parametrize("flags", [0, 2, 4, 6])
 def test_round_trip_and_stats_match_oracle(b, M, K, s, K_L, flags):
-    W = workloads.make_weight(M, K, s, seed=M + K, row_varying=(flags == 2))
+    W = workloads.make_weight(M, K, s, seed=M + K, row_varying=bool(flags & 2))
     h = b.us_encode(W, fmt=(16, K_L, 2, 1), flags=b.US_ENCODE_HOST_ONLY | flags)
     try:
         assert (b.us_decode(h) == W).all()
@@ -57,6 +57,20 @@ def test_round_trip_and_stats_match_oracle(b, M, K, s, K_L, flags):
         if flags == 2:   # rows ordered by nonzero count
             cnt = (Wp != 0).sum(1)[: M]
             assert (np.diff(cnt) >= 0).all()
+        if flags & 4:    # rows paired inside each strip (Alg. 1 on the 16 x K strip, R_A = 2, C_A = 1)
+            plain = b.us_encode(W, fmt=(16, K_L, 2, 1), flags=b.US_ENCODE_HOST_ONLY | (flags & 2))
+            base = b.us_get_row_order(plain)
+            plain_P = b.us_get_stats(plain)["sum_P"]
+            b.us_destroy(plain)
+            best = 0
+            for rb in range(st["Mp"] // 16):
+                # the same 16 rows as without the flag, in some other order
+                assert sorted(order[16 * rb: 16 * rb + 16]) == sorted(base[16 * rb: 16 * rb + 16])
+                rows = base[16 * rb: 16 * rb + 16]
+                strip = np.zeros((16, K), np.int8)
+                strip[rows >= 0] = W[rows[rows >= 0]]
+                best += oracle.reorder_tile(strip != 0, 2, 1)[1]
+            assert st["sum_P"] == best <= plain_P
     finally:
         b.us_destroy(h)
 

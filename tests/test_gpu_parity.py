@@ -68,9 +68,10 @@ def test_attention_4096(b, i, s):
 
 
 @pytest.mark.parametrize("M,K,seed", [(11008, 4096, 300), (4096, 11008, 302)])
-@pytest.mark.parametrize("flags", [0, 2])
+@pytest.mark.parametrize("flags", [0, 2, 4, 6])
 def test_ffn_7b_row_varying(b, M, K, seed, flags):
-    """Row-varying density (keep rate ~U(0.3, 0.7) per row), with and without the row order."""
+    """Row-varying density (keep rate ~U(0.3, 0.7) per row); flags: rows sorted by density (2),
+    rows paired inside each strip as Alg. 1 says (4), both (6)."""
     W = workloads.make_weight(M, K, 0.5, seed=seed, row_varying=True)
     X = workloads.make_x(K, 32, seed=seed)
     s_w, s_x = workloads.make_scales(M, 32, seed=seed)
