@@ -16,6 +16,7 @@ struct us_handle {
     int sm_count = 0;
     int max_N = 0;
     int max_smem = 0;
+    int co_warps = 10;   // warps of an N <= 8 CTA when two CTAs share an SM's registers
     uint8_t* d_blob = nullptr;
     uint32_t* d_item_off = nullptr;
     std::vector<uint32_t> cta_begin[4];  // schedule per N class (NT = 1, 2, 4, 8)
@@ -49,7 +50,7 @@ int local_acc_budget() { static int v = env_int("US_LOCAL_ACC_KB", 32) * 1024; r
 int stages_knob() { static int v = env_int("US_STAGES", 0); return v; }     // ring slots per warp, 0 = automatic
 int lut_rep_knob() { static int v = env_int("US_LUT_REP", 0); return v; }   // selector-table copies, 0 = automatic
 int pdl_knob() { static int v = env_int("US_PDL", 1); return v; }          // programmatic dependent launch
-int half_sm_knob() { static int v = env_int("US_HALF_SM", 0); return v; }  // small problems: half an SM per CTA
+int coresident_knob() { static int v = env_int("US_CORESIDENT", 1); return v; }  // small problems: half an SM per CTA
 int max_warps() { static int v = std::min(16, std::max(2, env_int("US_MAX_WARPS", 16))); return v; }
 
 struct LaunchGeom {
@@ -74,8 +75,11 @@ int segs_per_range(const us::HostMatrix& hm, int nt, int limit, int64_t min_rang
     const int slot = (int)((hm.max_item_bytes + 256u + 127u) & ~127u);
     const int acc = nt * 512 * 2 <= local_acc_budget() ? local_acc_budget() : 0;
     const int other = 256 * 8 * 4 + (int)us::kLutScratchBytes + acc + 2 * us::kOffTable * 4 + 1024;
-    const int want = std::min(max_warps(), min_warps_knob());
     for (int64_t r = std::max<int64_t>(1, min_ranges); r <= n_segs; ++r) {
+        // A single range is worth more (no partial sums leave the CTA when the cuts fall on strip
+        // boundaries): it may cost two more warps. Measured on 4096 x 11008, N = 8: one range with
+        // 15 warps 9.8 us, two ranges with 16 warps 14.7 us.
+        const int want = std::min(max_warps(), r == 1 ? std::min(10, min_warps_knob()) : min_warps_knob());
         const int64_t G = (n_segs + r - 1) / r;
         const int64_t xb = (int64_t)nt * 8 * (G * hm.fmt.K_L + 32) + G * nt * 32;
         if ((limit - other - xb) / slot >= want) return (int)G;
@@ -117,15 +121,21 @@ bool plan_launch(const us_handle* h, int N, LaunchGeom* g)
     }
     int stages = stages_knob() > 0 ? stages_knob() : (warps_for(1) >= warps_for(2) + 3 ? 1 : 2);
     int warps = warps_for(stages);
-    const int fixed = fixed_base + 32 * stages * 8;
     if (warps < kMinWarps) return false;
-    // Small problems (a CTA sees only a few tiles per warp): take at most half an SM -- shared
-    // memory and registers -- so that the next launch's CTA can move in beside this one and run its
-    // latency-bound prologue under this one's decode (programmatic dependent launch).
+    // Small problems at N <= 8 (a CTA sees about a tile per warp): take at most half an SM -- shared
+    // memory and registers -- with one slot per warp, so that the next launch's CTA moves in beside
+    // this one and runs its latency-bound prologue (parameters, offsets, first tile copies, table)
+    // under this one's work; with one CTA per SM, programmatic dependent launch alone hides only the
+    // launch latency, because all CTAs of a launch end at about the same time.
+    // Measured on 4096 x 4096, N = 8: 6.6 -> 5.7 us; not worth it from ~20 tiles per CTA on.
     const int64_t per_cta = (h->host.n_items + 147) / 148;
-    if (half_sm_knob() && per_cta <= 3 * (int64_t)warps) {
-        const int half = limit / 2 - 2048;
-        while (warps > 4 && (fixed + warps * stages * (int)g->slot_bytes > half || warps > 8)) --warps;
+    int fixed = fixed_base + 32 * stages * 8;
+    if (coresident_knob() && g->nt == 1 && per_cta <= 16 && stages_knob() == 0 && lut_rep_knob() == 0) {
+        const int half = 228 * 1024 / 2 - 1024 - 512;   // per SM: 228 KB, 1 KB reserved per CTA
+        const int fixed8 = fixed_for(8) + 32 * 8;
+        int w = std::min(h->co_warps, max_warps());
+        while (w >= 8 && fixed8 + w * (int)g->slot_bytes > half) --w;
+        if (w >= 8) { stages = 1; lut_rep = 8; warps = w; fixed = fixed8; }
     }
     g->stages = stages;
     g->lut_rep = lut_rep;
@@ -275,6 +285,18 @@ us_status us_encode(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_sca
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device);
     if (e == cudaSuccess && h->sm_count > us::kMaxCtas) h->sm_count = us::kMaxCtas;
     if (e == cudaSuccess) e = enable_large_smem(h->max_smem);
+    if (e == cudaSuccess) {
+        // Two N <= 8 CTAs share the SM's 64 K registers (allocated 8 per thread at a time).
+        int regs = 0;
+        // (the stage-timer builds need more and simply do not share an SM)
+        for (const void* f : {(const void*)us::us_spmm_kernel<1, 1, true, false>, (const void*)us::us_spmm_kernel<1, 1, false, false>}) {
+            cudaFuncAttributes fa;
+            e = cudaFuncGetAttributes(&fa, f);
+            if (e != cudaSuccess) break;
+            regs = std::max(regs, fa.numRegs);
+        }
+        if (e == cudaSuccess) h->co_warps = 32768 / (32 * ((regs + 7) / 8 * 8));
+    }
     if (e != cudaSuccess) { delete h; return US_ERR_CUDA; }
 
     const us::HostMatrix& hm = h->host;

@@ -284,14 +284,31 @@ struct StoreCtx {   // what the store needs, by value (the full parameter block 
     uint32_t* cnt;
     int32_t M, N, fp16_out;
 };
+// Scales fetched ahead of the store (fp16 output): the two weight scales of a lane's rows of one
+// strip, and (small N only) the activation scales of the lane's tokens.
 template <int NT>
-__device__ __forceinline__ void store_rows(const StoreCtx p, const int (&v)[NT][4], int lane, int m_lo, int m_hi)
+struct ScalePre {
+    static constexpr bool kSx = NT <= 2;
+    int rb = -1;                 // strip the weight scales belong to (-1 = none)
+    // raw fp16 bit patterns: converting at the point of use keeps the loads in flight meanwhile
+    unsigned short sw_lo = 0, sw_hi = 0;
+    bool have_sx = false;
+    unsigned short sx[kSx ? NT : 1][2];
+};
+template <int NT>
+__device__ __forceinline__ void store_rows(const StoreCtx p, const int (&v)[NT][4], int lane, int m_lo, int m_hi,
+                                           const ScalePre<NT>* pre = nullptr, int rb = -2)
 {
     const int t2 = (lane & 3) * 2;
     float sw_lo = 0.f, sw_hi = 0.f;
     if (p.fp16_out) {
-        if (m_lo >= 0) sw_lo = __half2float(__ushort_as_half(__ldg(p.w_scale + m_lo)));
-        if (m_hi >= 0) sw_hi = __half2float(__ushort_as_half(__ldg(p.w_scale + m_hi)));
+        if (pre && pre->rb == rb) {
+            sw_lo = __half2float(__ushort_as_half(pre->sw_lo));
+            sw_hi = __half2float(__ushort_as_half(pre->sw_hi));
+        } else {
+            if (m_lo >= 0) sw_lo = __half2float(__ushort_as_half(__ldg(p.w_scale + m_lo)));
+            if (m_hi >= 0) sw_hi = __half2float(__ushort_as_half(__ldg(p.w_scale + m_hi)));
+        }
     }
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt)
@@ -302,7 +319,9 @@ __device__ __forceinline__ void store_rows(const StoreCtx p, const int (&v)[NT][
             if (n >= p.N || m < 0) continue;
             const size_t o = (size_t)n * p.M + m;
             if (p.fp16_out) {
-                const float sx = __half2float(__ushort_as_half(__ldg(p.x_scale + n)));
+                float sx;
+                if (ScalePre<NT>::kSx && pre && pre->have_sx) sx = __half2float(__ushort_as_half(pre->sx[ScalePre<NT>::kSx ? nt : 0][j & 1]));
+                else sx = __half2float(__ushort_as_half(__ldg(p.x_scale + n)));
                 const float r = (float)v[nt][j] * ((j < 2) ? sw_lo : sw_hi) * sx;
                 reinterpret_cast<__half*>(p.Y)[o] = __float2half_rn(r);
             } else {
@@ -525,6 +544,13 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
     uint32_t item[STAGES];        // position u held (or awaited) by each ring slot
     uint32_t ahead;               // next position, whose offsets are already being fetched
     uint32_t po0 = 0, po1 = 0;    // its offsets (valid in lane 0)
+    int pre_rb = -1, pre_mlo = -1, pre_mhi = -1;   // fp16 output: rows of the warp's first strip
+    if (p.fp16_out && static_pos(0) < end) {
+        int kr0, sg0;
+        tile_of(static_pos(0), kr0, pre_rb, sg0);
+        pre_mlo = __ldg(p.row_order + pre_rb * 16 + (lane >> 2));
+        pre_mhi = __ldg(p.row_order + pre_rb * 16 + (lane >> 2) + 8);
+    }
     {
         // lanes 0..STAGES fetch the offsets of the first STAGES+1 positions in parallel
         const uint32_t mine = static_pos(lane <= STAGES ? lane : 0);
@@ -597,12 +623,43 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
     // Everything above (schedule, offsets, selector table, the first weight-tile copies) depends on
     // nothing an earlier kernel of the stream produces. X may be the output of the kernel before,
     // and Y / the workspace may still be in use by it: wait for the stream's earlier work here.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    // The activations of the CTA's first K range: fetch them into registers now, ahead of the
-    // staging pass.
     int kr_first, kr_last, d0_, d1_;
     tile_of(beg, kr_first, d0_, d1_);
     tile_of(end - 1, kr_last, d0_, d1_);
+    // Still independent of the stream's earlier work: the weight scales of the rows of this warp's
+    // first strip (any warp may be the one that stores it; their row numbers were requested together
+    // with the first offsets), the cleared sums and the table copies.
+    ScalePre<NT> spre;
+    if (pre_rb >= 0) {
+        if (pre_mlo >= 0) spre.sw_lo = __ldg(p.w_scale + pre_mlo);
+        if (pre_mhi >= 0) spre.sw_hi = __ldg(p.w_scale + pre_mhi);
+        spre.rb = pre_rb;
+    }
+    auto clear_sums = [&]() {
+        for (int i = threadIdx.x; i < p.G * NT * 8; i += blockDim.x) sx16[i] = 0;
+        if (LA) {
+            for (int i = threadIdx.x; i < p.s_local * NT * 128; i += blockDim.x) acc_l[i] = 0;
+            for (int i = threadIdx.x; i < p.s_local; i += blockDim.x) cnt_l[i] = 0;
+        }
+        __syncthreads();
+    };
+    clear_sums();
+    // copies of the selector table: entry e, copy r at word e * lut_rep + r (conflict-free writes)
+    for (int i = threadIdx.x, sh = 31 - __clz(p.lut_rep); i < 256 * p.lut_rep; i += blockDim.x) lut[i] = lut1[i >> sh];
+
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // The activations of the CTA's first K range: fetch them into registers now, ahead of the
+    // staging pass; and the activation scales of this lane's tokens.
+    if (ScalePre<NT>::kSx && p.fp16_out) {
+#pragma unroll
+        for (int nt = 0; nt < (ScalePre<NT>::kSx ? NT : 1); ++nt)
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const int n = nt * 8 + (lane & 3) * 2 + j;
+                spre.sx[nt][j] = n < p.N ? __ldg(p.x_scale + n) : (unsigned short)0;
+            }
+        spre.have_sx = true;
+    }
     const int g_first = (kr_first == n_kr - 1) ? g_last : p.G;   // segments in that range
     constexpr int kXPre = NT == 1 ? 8 : NT == 2 ? 4 : 0;   // 16-byte units of X a thread prefetches
     const int x_sh = 31 - __clz(p.K_L / 32);   // log2(units per (segment, token)) when a power of two
@@ -637,7 +694,7 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
             m_lo = __ldg(p.row_order + rb * 16 + (lane >> 2));
             m_hi = __ldg(p.row_order + rb * 16 + (lane >> 2) + 8);
         }
-        store_rows<NT>(sctx, v, lane, m_lo, m_hi);
+        store_rows<NT>(sctx, v, lane, m_lo, m_hi, &spre, rb);
     };
     // add v to the global workspace of strip rb
     auto red_global = [&](int rb, int (&v)[NT][4]) {
@@ -673,15 +730,9 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
     for (int nt = 0; nt < NT; ++nt) y[nt][0] = y[nt][1] = y[nt][2] = y[nt][3] = 0;
 
     // Stage the activations of K range kr: clear the sums, expand X, synchronise.
-    auto stage_range = [&](int kr, int g_kr, bool use_prefetched) {
-        for (int i = threadIdx.x; i < p.G * NT * 8; i += blockDim.x) sx16[i] = 0;
-        if (LA) {
-            for (int i = threadIdx.x; i < p.s_local * NT * 128; i += blockDim.x) acc_l[i] = 0;
-            for (int i = threadIdx.x; i < p.s_local; i += blockDim.x) cnt_l[i] = 0;
-        }
-        __syncthreads();
-        // copies of the selector table: entry e, copy r at word e * lut_rep + r (conflict-free writes)
-        for (int i = threadIdx.x, sh = 31 - __clz(p.lut_rep); i < 256 * p.lut_rep; i += blockDim.x) lut[i] = lut1[i >> sh];
+    auto stage_range = [&](int kr, int g_kr, bool first) {
+        const bool use_prefetched = first && x_early;
+        if (!first) clear_sums();
         if (use_prefetched) {
             // expand the prefetched units; anything beyond them goes through the general path
 #pragma unroll
@@ -718,7 +769,7 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
 #endif
     // The first range is staged here, outside the loop, so that the prefetched X registers are
     // dead before the decode loop starts.
-    stage_range(kr_first, g_first, x_early);
+    stage_range(kr_first, g_first, true);
 #ifndef US_EXP_EPI_TIMERS
     if (timing) dbg[3] = clock64() - t_start;
 #endif
