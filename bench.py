@@ -332,7 +332,7 @@ def run_ours(args, rank: int, local_rank: int, world: int):
                      "unit": "GB/s", "frac": alg / per_launch / 1e9 / peak_gbs, "peak_kind": peak_kind,
                      "traffic": TRAFFIC_BYTES_PER_LAUNCH, "algorithmic_bytes": alg,
                      "stored_bytes": binding.us_spmm_bytes(head.sw[0].handle, N, True),
-                     "kernel": "us_spmm_kernel<1,2,1,1> on 4096x4096 s=0.5 N=8 fp16"},
+                     "kernel": kernel_label(binding, head.sw[0].handle, N) + " on 4096x4096 s=0.5 N=8 fp16"},
         "stats": {k: head.stats[k] for k in ("nnz", "sum_P", "bytes_payload", "bytes_payload_padded",
                                              "bytes_bitmap", "bytes_offsets", "pmr", "fill")},
     }
@@ -347,13 +347,20 @@ def run_ours(args, rank: int, local_rank: int, world: int):
                                      "frac": r["gbs"] / peak_gbs, "pct_of_8tbs": r["pct_of_8tbs"],
                                      "us": r["us"], "algorithmic_bytes": r["alg_bytes"],
                                      "traffic": 102_084_864,   # profiles/us_spmm_kernel_28672x8192_s60_n8_int32.md
-                                     "kernel": "us_spmm_kernel<1,2,1,1> on 28672x8192 s=0.6 N=8 int32"}
+                                     "kernel": r["kernel"] + " on 28672x8192 s=0.6 N=8 int32"}
     if rank == 0:
         out["cpu_baseline"] = cpu_baseline(W, Xall[:N], s_w, s_x[:N], pstats)
         print(json.dumps(out))
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def kernel_label(binding, handle, N):
+    """The dominant (only) kernel of a call and its launch geometry."""
+    g = binding.us_launch_info(handle, N)
+    return (f"us_spmm_kernel (n-tiles {max(1, 1 << (max(N, 1) - 1).bit_length()) // 8 or 1}, {g['grid']} CTAs x "
+            f"{g['block'] // 32} warps, {g['smem_bytes']} B shared memory)")
 
 
 # Measured DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the
@@ -384,7 +391,7 @@ def sweep(binding, torch, workloads, l2, peak_gbs):
                          "gbs": alg / t / 1e9, "pct_of_8tbs": 100 * alg / t / 1e9 / CONTRACT_PEAK_GBS,
                          "frac_of_measured": alg / t / 1e9 / peak_gbs,
                          "dense_equiv_tops": 2.0 * M * K * N / t / 1e12, "replicas": R,
-                         "pmr": case.stats["pmr"]})
+                         "pmr": case.stats["pmr"], "kernel": kernel_label(binding, case.sw[0].handle, N)})
         case.close()
         del case
         torch.cuda.empty_cache()
