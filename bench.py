@@ -281,23 +281,45 @@ def run_ours(args, rank: int, local_rank: int, world: int):
     value = alg * launches * world / dt / 1e9
 
     # ---- end to end: host buffers, H2D of X and scales, D2H of Y inside the timed region --------
-    Xh = head.Xh[:N].clone().pin_memory()
-    sxh = torch.from_numpy(s_x[:N].copy()).pin_memory()
-    Yh = torch.empty((N, HEAD["M"]), dtype=torch.float16).pin_memory()
-    Xd = torch.empty_like(Xh, device="cuda")
-    sxd = torch.empty_like(sxh, device="cuda")
-    Yd = torch.empty((N, HEAD["M"]), dtype=torch.float16, device="cuda")
+    # One step = R SpMMs, each with its own (X | activation scales) block in pinned host memory and
+    # its own Y block: one batched copy in, the R library calls, one batched copy of all results
+    # back to pinned host memory. The step is captured once as a CUDA graph -- the copies are memcpy
+    # nodes that read / write the host buffers at every replay.
+    x_bytes = head.Xh[:N].numel()
+    sx_off = (x_bytes + 15) // 16 * 16
+    blk = (sx_off + 2 * N + 255) // 256 * 256
+    in_h = torch.zeros((R, blk), dtype=torch.uint8).pin_memory()
+    in_h[:, :x_bytes] = head.Xh[:N].reshape(-1)
+    in_h[:, sx_off:sx_off + 2 * N] = torch.from_numpy(s_x[:N].copy()).view(torch.uint8)
+    in_d = torch.empty_like(in_h, device="cuda")
+    Yh = torch.empty((R, N, HEAD["M"]), dtype=torch.float16).pin_memory()
+    Yd = torch.empty((R, N, HEAD["M"]), dtype=torch.float16, device="cuda")
+
+    def e2e_enqueue():
+        in_d.copy_(in_h, non_blocking=True)
+        for r, sw in enumerate(head.sw):
+            sw.spmm(in_d[r, :x_bytes].view(N, -1), N, in_d[r, sx_off:sx_off + 2 * N].view(torch.float16), out=Yd[r])
+        Yh.copy_(Yd, non_blocking=True)
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        e2e_enqueue()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    e2e_graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(e2e_graph):
+        e2e_enqueue()
 
     def e2e_step():
-        for sw in head.sw:
-            Xd.copy_(Xh, non_blocking=True)
-            sxd.copy_(sxh, non_blocking=True)
-            sw.spmm(Xd, N, sxd, out=Yd)
-            Yh.copy_(Yd, non_blocking=True)
-        torch.cuda.synchronize()
+        e2e_graph.replay()
+        torch.cuda.synchronize()   # the step's results are in host memory from here on
 
     for _ in range(3):
         e2e_step()
+    ref16 = head.Y16[:N].cpu()   # every replica holds the same W and gets the same X: same Y
+    if not all(torch.equal(Yh[r], ref16) for r in range(R)):
+        raise RuntimeError("end-to-end result differs from the device-resident run")
     e2e_steps = max(3, min(args.steps, 50))
     barrier()
     t0 = time.perf_counter()
@@ -305,8 +327,8 @@ def run_ours(args, rank: int, local_rank: int, world: int):
         e2e_step()
     t_e2e = max_over_ranks(time.perf_counter() - t0, dist, "cuda")
     e2e_value = alg * R * e2e_steps * world / t_e2e / 1e9
-    h2d = R * (Xh.numel() + sxh.numel() * 2)
-    d2h = R * Yh.numel() * 2
+    h2d = in_h.numel()
+    d2h = Yh.numel() * 2
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
