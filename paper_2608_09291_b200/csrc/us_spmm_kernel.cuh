@@ -545,7 +545,10 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
     uint32_t ahead;               // next position, whose offsets are already being fetched
     uint32_t po0 = 0, po1 = 0;    // its offsets (valid in lane 0)
     int pre_rb = -1, pre_mlo = -1, pre_mhi = -1;   // fp16 output: rows of the warp's first strip
-    if (p.fp16_out && static_pos(0) < end) {
+    // (Only the N <= 16 kernels fetch scales ahead: the wider ones have no registers to spare --
+    // measured at N = 64 on a 28672 x 8192 matrix: 102 us with this code compiled in, 87 us without.)
+    constexpr bool kPreScales = NT <= 2;
+    if (kPreScales && p.fp16_out && static_pos(0) < end) {
         int kr0, sg0;
         tile_of(static_pos(0), kr0, pre_rb, sg0);
         pre_mlo = __ldg(p.row_order + pre_rb * 16 + (lane >> 2));
@@ -630,7 +633,7 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
     // first strip (any warp may be the one that stores it; their row numbers were requested together
     // with the first offsets), the cleared sums and the table copies.
     ScalePre<NT> spre;
-    if (pre_rb >= 0) {
+    if (kPreScales && pre_rb >= 0) {
         if (pre_mlo >= 0) spre.sw_lo = __ldg(p.w_scale + pre_mlo);
         if (pre_mhi >= 0) spre.sw_hi = __ldg(p.w_scale + pre_mhi);
         spre.rb = pre_rb;
@@ -650,7 +653,7 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
     asm volatile("griddepcontrol.wait;" ::: "memory");
     // The activations of the CTA's first K range: fetch them into registers now, ahead of the
     // staging pass; and the activation scales of this lane's tokens.
-    if (ScalePre<NT>::kSx && p.fp16_out) {
+    if (kPreScales && ScalePre<NT>::kSx && p.fp16_out) {
 #pragma unroll
         for (int nt = 0; nt < (ScalePre<NT>::kSx ? NT : 1); ++nt)
 #pragma unroll
@@ -694,7 +697,7 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
             m_lo = __ldg(p.row_order + rb * 16 + (lane >> 2));
             m_hi = __ldg(p.row_order + rb * 16 + (lane >> 2) + 8);
         }
-        store_rows<NT>(sctx, v, lane, m_lo, m_hi, &spre, rb);
+        store_rows<NT>(sctx, v, lane, m_lo, m_hi, kPreScales ? &spre : nullptr, rb);
     };
     // add v to the global workspace of strip rb
     auto red_global = [&](int rb, int (&v)[NT][4]) {
