@@ -22,6 +22,7 @@ struct us_handle {
     std::vector<uint32_t> cta_begin[4];  // schedule per N class (NT = 1, 2, 4, 8)
     int G[4] = {1, 1, 1, 1};          // segments per K range, per class
     int s_local[4] = {0, 0, 0, 0};    // strips held in shared memory (0 = direct mode), per class
+    bool xp[4] = {false, false, false, false};   // X staged packed (half the shared memory), per class
     int32_t* d_row_order = nullptr;
     uint16_t* d_w_scale = nullptr;
     int32_t* d_acc = nullptr;
@@ -56,6 +57,7 @@ int max_warps() { static int v = std::min(16, std::max(2, env_int("US_MAX_WARPS"
 struct LaunchGeom {
     int nt, cls, warps, stages, smem, lut_rep;
     uint32_t slot_bytes;
+    bool xp;
 };
 
 // Segments per K range for an N class. The int8 activations of one K range live in shared memory
@@ -63,9 +65,17 @@ struct LaunchGeom {
 // Returns the range length of the split into the fewest equal ranges, not fewer than min_ranges,
 // that still leaves room for min_warps one-slot warps (measured: 15 warps and one range beat
 // 16 warps and two ranges by 25 % on a 13824 x 5120 matrix at N = 16).
+int xp_knob() { static int v = env_int("US_PACKED_X", 1); return v; }   // 0 off, 1 automatic, 2 whenever possible
 bool plan_debug() { static int v = env_int("US_PLAN_DEBUG", 0); return v != 0; }
 int min_warps_knob() { static int v = env_int("US_MIN_WARPS", 12); return v; }
-int segs_per_range(const us::HostMatrix& hm, int nt, int limit, int64_t min_ranges)
+// Shared memory of one K range's activations: int8 (one byte per token and k, 32 bytes of pad per
+// token row) or packed (half of that).
+int64_t x_bytes(int nt, int64_t G, int K_L, bool xp)
+{
+    return xp ? (int64_t)nt * 8 * (G * K_L / 2 + 16) : (int64_t)nt * 8 * (G * K_L + 32);
+}
+
+int segs_per_range(const us::HostMatrix& hm, int nt, int limit, int64_t min_ranges, bool xp)
 {
     const int64_t n_segs = hm.n_segs;
     if (x_budget() > 0) {
@@ -81,7 +91,7 @@ int segs_per_range(const us::HostMatrix& hm, int nt, int limit, int64_t min_rang
         // 15 warps 9.8 us, two ranges with 16 warps 14.7 us.
         const int want = std::min(max_warps(), r == 1 ? std::min(10, min_warps_knob()) : min_warps_knob());
         const int64_t G = (n_segs + r - 1) / r;
-        const int64_t xb = (int64_t)nt * 8 * (G * hm.fmt.K_L + 32) + G * nt * 32;
+        const int64_t xb = x_bytes(nt, G, hm.fmt.K_L, xp) + G * nt * 32;
         if ((limit - other - xb) / slot >= want) return (int)G;
     }
     return 1;
@@ -94,11 +104,12 @@ bool plan_launch(const us_handle* h, int N, LaunchGeom* g)
     g->nt = nt_for(N);
     g->cls = class_of(g->nt);
     const int G = h->G[g->cls], s_local = h->s_local[g->cls];
+    g->xp = h->xp[g->cls];
     g->slot_bytes = (h->host.max_item_bytes + 256u + 127u) & ~127u;
     // selector table copies: 32 (conflict-free lookups) when that costs no warp, else 8
     int lut_rep = 32;
     auto fixed_for = [&](int rep) {
-        return 256 * rep * 4 + (int)us::kLutScratchBytes + g->nt * 8 * (G * h->host.fmt.K_L + 32) + G * g->nt * 8 * 4 +
+        return 256 * rep * 4 + (int)us::kLutScratchBytes + (int)x_bytes(g->nt, G, h->host.fmt.K_L, g->xp) + G * g->nt * 8 * 4 +
                            32 * 4 + s_local * (g->nt * 128 + 1) * 4 + 2 * us::kOffTable * 4 + 128;
     };
     int fixed_base = fixed_for(lut_rep);
@@ -144,7 +155,8 @@ bool plan_launch(const us_handle* h, int N, LaunchGeom* g)
     return true;
 }
 
-// Chooses, per N class, the K-range width and whether strips are summed in shared memory.
+// Chooses, per N class, the K-range width, whether strips are summed in shared memory, and whether
+// X is staged packed.
 void plan_classes(us_handle* h, int n_cta, std::vector<uint32_t> (&sched)[4])
 {
     const int limit = h->max_smem > 0 ? h->max_smem : 227 * 1024;
@@ -152,32 +164,58 @@ void plan_classes(us_handle* h, int n_cta, std::vector<uint32_t> (&sched)[4])
         const int nt = 1 << c;
         // Local mode needs the strip sums of a CTA's share of one K range in shared memory; a short
         // last range spreads a CTA over more strips, so shorter ranges are tried before giving up.
+        // Returns the range length found (0 = none) and leaves the schedule in `out`.
+        auto local_plan = [&](bool xp, std::vector<uint32_t>* out, int* s_local) -> int {
+            int G = 0, worst = 1;
+            for (int64_t r = 1; r <= h->host.n_segs; ++r) {
+                const int Gr = segs_per_range(h->host, nt, limit, r, xp);
+                if (Gr == G) continue;
+                G = Gr;
+                if (G <= 1) break;
+                us::make_schedule(h->host, n_cta, G, out, &worst);
+                if (plan_debug())
+                    fprintf(stderr, "[unionsparse] plan nt=%d%s: G=%d needs %d local strips\n", nt, xp ? " packed X" : "", G, worst);
+                if (worst * nt * 512 <= local_acc_budget()) { *s_local = worst; return G; }
+            }
+            return 0;
+        };
         h->G[c] = 1;
         h->s_local[c] = 0;
-        int G = 0, worst = 1;
-        for (int64_t r = 1; r <= h->host.n_segs; ++r) {
-            const int Gr = segs_per_range(h->host, nt, limit, r);
-            if (Gr == G) continue;
-            G = Gr;
-            if (G <= 1) break;
-            us::make_schedule(h->host, n_cta, G, &sched[c], &worst);
-            if (plan_debug())
-                fprintf(stderr, "[unionsparse] plan nt=%d: G=%d needs %d local strips\n", nt, G, worst);
-            if (worst * nt * 512 <= local_acc_budget()) {
-                h->G[c] = G;
-                h->s_local[c] = worst;
-                break;
+        h->xp[c] = false;
+        int sl = 0;
+        const int G = local_plan(false, &sched[c], &sl);
+        if (G > 0) { h->G[c] = G; h->s_local[c] = sl; }
+        // Packed X (N = 9..16 only: the kernel exists for that class) halves the shared memory of a
+        // K range at the price of three more integer instructions per n-tile and k-block. Worth it
+        // when it turns several K ranges into one (then no partial sum leaves the CTA).
+        // Measured at N = 16: 28672 x 8192 38.4 -> 34.8 us and 4096 x 11008 17.9 -> 14.4 us (two
+        // ranges become one); 5120 x 5120 12.0 -> 9.4 us (one range either way, but a CTA's share is
+        // small and the staging pass and the freed shared memory count for more than the decode);
+        // 13824 x 5120 15.7 -> 16.0 us (one range either way, long decode): not taken there.
+        if (nt == 2 && xp_knob() != 0) {
+            const int64_t n_segs = h->host.n_segs;
+            const int64_t ranges = (n_segs + h->G[c] - 1) / h->G[c];
+            const bool small_share = (int64_t)h->host.blob.size() / std::max(1, n_cta) < 128 * 1024;
+            if (ranges > 1 || small_share || xp_knob() == 2) {
+                std::vector<uint32_t> alt;
+                int sl2 = 0;
+                const int G2 = local_plan(true, &alt, &sl2);
+                if (G2 > 0 && ((n_segs + G2 - 1) / G2 == 1 || xp_knob() == 2)) {
+                    h->G[c] = G2; h->s_local[c] = sl2; h->xp[c] = true;
+                    sched[c] = alt;
+                }
             }
         }
         // direct mode: one segment per range, every tile goes to the global workspace (longer ranges
         // and runs were measured: no gain at N = 32, the bigger X costs more than the adds it saves)
+        int worst = 1;
         if (h->s_local[c] == 0) us::make_schedule(h->host, n_cta, 1, &sched[c], &worst);
     }
 }
 
 int run_knob() { static int v = env_int("US_RUN", 0); return v; }
 template <int NT, int ST>
-cudaError_t launch_st(const us::SpmmParams& p, int grid, int block, int smem, cudaStream_t st)
+cudaError_t launch_st(const us::SpmmParams& p, bool xp, int grid, int block, int smem, cudaStream_t st)
 {
     // Launched with programmatic stream serialization: the kernel may start while its predecessor
     // in the stream is still running; it waits (griddepcontrol.wait) before it touches anything
@@ -193,6 +231,9 @@ cudaError_t launch_st(const us::SpmmParams& p, int grid, int block, int smem, cu
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     const bool la = p.s_local > 0, timed = p.timers != nullptr;
+    if (NT == 2 && xp && la)   // packed X: planned for this class and local mode only
+        return timed ? cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<2, ST, true, true, true>, p)
+                     : cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<2, ST, true, false, true>, p);
     if (la && !timed) return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, ST, true, false>, p);
     if (!la && !timed) return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, ST, false, false>, p);
     if (la) return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, ST, true, true>, p);
@@ -200,9 +241,9 @@ cudaError_t launch_st(const us::SpmmParams& p, int grid, int block, int smem, cu
 }
 
 template <int NT>
-cudaError_t launch_nt(const us::SpmmParams& p, int stages, int grid, int block, int smem, cudaStream_t st)
+cudaError_t launch_nt(const us::SpmmParams& p, bool xp, int stages, int grid, int block, int smem, cudaStream_t st)
 {
-    return stages == 1 ? launch_st<NT, 1>(p, grid, block, smem, st) : launch_st<NT, 2>(p, grid, block, smem, st);
+    return stages == 1 ? launch_st<NT, 1>(p, xp, grid, block, smem, st) : launch_st<NT, 2>(p, xp, grid, block, smem, st);
 }
 
 // Opt every kernel variant in to the device's full dynamic shared memory (once per handle, at
@@ -230,6 +271,11 @@ cudaError_t enable_large_smem(int bytes)
     if (e == cudaSuccess) e = enable_large_smem_nt<2>(bytes);
     if (e == cudaSuccess) e = enable_large_smem_nt<4>(bytes);
     if (e == cudaSuccess) e = enable_large_smem_nt<8>(bytes);
+    const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<2, 1, true, false, true>, attr, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<2, 2, true, false, true>, attr, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<2, 1, true, true, true>, attr, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<2, 2, true, true, true>, attr, bytes);
     return e;
 }
 
@@ -411,10 +457,10 @@ us_status us_spmm(us_handle* h, const void* X, int32_t N, const void* x_scale, v
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e;
     switch (g.nt) {
-        case 1: e = launch_nt<1>(p, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
-        case 2: e = launch_nt<2>(p, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
-        case 4: e = launch_nt<4>(p, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
-        default: e = launch_nt<8>(p, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
+        case 1: e = launch_nt<1>(p, g.xp, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
+        case 2: e = launch_nt<2>(p, g.xp, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
+        case 4: e = launch_nt<4>(p, g.xp, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
+        default: e = launch_nt<8>(p, g.xp, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
     }
     if (e != cudaSuccess) { h->sticky = e; return US_ERR_CUDA; }
     return US_OK;
@@ -493,10 +539,10 @@ us_status us_spmm_static_scratch(us_handle* h, const void* X, int32_t N, const v
     p.x_fast = (hm.K % 32 == 0) ? 2 : (hm.K % 8 == 0) ? 1 : 0;
     p.fp16_out = x_scale ? 1 : 0;
     switch (g.nt) {
-        case 1: e = launch_nt<1>(p, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
-        case 2: e = launch_nt<2>(p, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
-        case 4: e = launch_nt<4>(p, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
-        default: e = launch_nt<8>(p, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
+        case 1: e = launch_nt<1>(p, g.xp, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
+        case 2: e = launch_nt<2>(p, g.xp, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
+        case 4: e = launch_nt<4>(p, g.xp, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
+        default: e = launch_nt<8>(p, g.xp, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
     }
     if (e != cudaSuccess) { h->sticky = e; return US_ERR_CUDA; }
     return US_OK;

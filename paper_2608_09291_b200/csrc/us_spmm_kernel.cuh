@@ -199,9 +199,19 @@ __device__ __forceinline__ uint2 expand8(uint32_t v, int32_t& s)
     return make_uint2(prmt(te, to, 0x5140), prmt(te, to, 0x7362));
 }
 
+// Packed staging (XP): the same 8 activations as one word q whose even nibbles are k 0..3 and odd
+// nibbles k 4..7, so that the decode loop gets its two B-fragment words (x16, as int8) with
+// (q << 4) & 0xF0F0F0F0 and q & 0xF0F0F0F0. Half the shared memory of the int8 form for three more
+// integer instructions per n-tile and k-block.
+__device__ __forceinline__ uint32_t pack8(uint32_t v, int32_t& s)
+{
+    const uint2 t = expand8(v, s);
+    return (t.x >> 4) | t.y;
+}
+
 // sx16 must be zero on entry (the caller clears it and synchronises).
 // Units below `first_unit` (of the 16-byte path) were already staged by the caller.
-template <int NT>
+template <int NT, bool XP>
 __device__ __forceinline__ void stage_x(const SpmmParams& p, int seg0, int n_seg, uint8_t* x8,
                                         int xstride, int32_t* sx16, int first_unit)
 {
@@ -233,14 +243,21 @@ __device__ __forceinline__ void stage_x(const SpmmParams& p, int seg0, int n_seg
                     const int pi = u / upr, q = u - pi * upr;
                     const int sgl = pi / rows, n = pi - sgl * rows;
                     int32_t s = 0;
-                    uint4 lo, hi;
-                    uint2 t;
-                    t = expand8(v[b].x, s); lo.x = t.x; lo.y = t.y;
-                    t = expand8(v[b].y, s); lo.z = t.x; lo.w = t.y;
-                    t = expand8(v[b].z, s); hi.x = t.x; hi.y = t.y;
-                    t = expand8(v[b].w, s); hi.z = t.x; hi.w = t.y;
-                    uint4* dst = reinterpret_cast<uint4*>(x8 + n * xstride + sgl * p.K_L + 32 * q);
-                    dst[0] = lo; dst[1] = hi;
+                    if (XP) {
+                        uint4 pk;
+                        pk.x = pack8(v[b].x, s); pk.y = pack8(v[b].y, s);
+                        pk.z = pack8(v[b].z, s); pk.w = pack8(v[b].w, s);
+                        *reinterpret_cast<uint4*>(x8 + n * xstride + (sgl * p.K_L + 32 * q) / 2) = pk;
+                    } else {
+                        uint4 lo, hi;
+                        uint2 t;
+                        t = expand8(v[b].x, s); lo.x = t.x; lo.y = t.y;
+                        t = expand8(v[b].y, s); lo.z = t.x; lo.w = t.y;
+                        t = expand8(v[b].z, s); hi.x = t.x; hi.y = t.y;
+                        t = expand8(v[b].w, s); hi.z = t.x; hi.w = t.y;
+                        uint4* dst = reinterpret_cast<uint4*>(x8 + n * xstride + sgl * p.K_L + 32 * q);
+                        dst[0] = lo; dst[1] = hi;
+                    }
                     if (s) atomicAdd(sx16 + pi, s);
                 }
             }
@@ -269,7 +286,8 @@ __device__ __forceinline__ void stage_x(const SpmmParams& p, int seg0, int n_seg
             }
         }
         int32_t s = 0;
-        *reinterpret_cast<uint2*>(x8 + n * xstride + sgl * p.K_L + 8 * wi) = expand8(v, s);
+        if (XP) *reinterpret_cast<uint32_t*>(x8 + n * xstride + (sgl * p.K_L + 8 * wi) / 2) = pack8(v, s);
+        else *reinterpret_cast<uint2*>(x8 + n * xstride + sgl * p.K_L + 8 * wi) = expand8(v, s);
         if (s) atomicAdd(sx16 + pi, s);
     }
 }
@@ -339,7 +357,8 @@ __device__ __forceinline__ void store_rows(const StoreCtx p, const int (&v)[NT][
 // CH independent chains walk consecutive ranges of the tile's mask words.
 // All addresses are 32-bit shared-memory addresses: slot_a = the staged tile, lut_a = selector
 // table + 4*lane, xb_a = this lane's first B-fragment of the tile's segment.
-template <int NT, int CH>
+// XP: X is staged packed (one word per lane, k-block and n-tile) instead of as int8 (two words).
+template <int NT, int CH, bool XP>
 __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, uint32_t lut_stride,
                                              uint32_t xb_a, int xstride, int mask_rows, int lane,
                                              int (&c)[NT][4])
@@ -348,6 +367,14 @@ __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, ui
     const uint32_t mask_a = slot_a + 4u * lane;
     const uint32_t pay_a = slot_a + 128u * mask_rows + 4u * lane;
     constexpr bool kPreX = NT <= 2;   // small N: fetch the X fragments together with the windows
+    constexpr uint32_t kXStep = XP ? 16u : 32u;   // bytes of a token's row per k-block
+    auto ldx = [&](uint32_t a) -> uint2 {         // the lane's two B-fragment words at address a
+        if (XP) {
+            const uint32_t q = lds32(a);
+            return make_uint2((q * 16u) & 0xF0F0F0F0u, q & 0xF0F0F0F0u);
+        }
+        return lds64(a);
+    };
     uint32_t b8[CH];       // 8 * (byte position in the lane's payload stream), per chain
     uint32_t cw0[CH], cw1[CH];   // carried window: the two words at / after the chain's position
     b8[0] = 0;
@@ -390,7 +417,7 @@ __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, ui
                 if (kPreX) {
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt)
-                        xf[ch][i][nt] = lds64(xb_a + 32u * (4 * (ch * rows_per + w) + i) + nt * 8 * xstride);
+                        xf[ch][i][nt] = ldx(xb_a + kXStep * (4 * (ch * rows_per + w) + i) + nt * 8 * xstride);
                 }
             }
 #pragma unroll
@@ -408,7 +435,7 @@ __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, ui
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
                     const uint2 b = kPreX ? xf[ch][i][nt]
-                                          : lds64(xb_a + 32u * (4 * (ch * rows_per + w) + i) + nt * 8 * xstride);
+                                          : ldx(xb_a + kXStep * (4 * (ch * rows_per + w) + i) + nt * 8 * xstride);
                     mma_s8(c[nt], d0, e0, d1, e1, b.x, b.y);
                 }
             }
@@ -446,7 +473,7 @@ __device__ __forceinline__ uint32_t fdiv(uint32_t u, unsigned long long m)
 // LA = local mode (shared-memory strip accumulators), else direct mode.
 // TIMED = record the diagnostic stage timers (a separate instantiation, so that the production
 // kernel carries none of their clock reads and branches).
-template <int NT, int STAGES, bool LA, bool TIMED>
+template <int NT, int STAGES, bool LA, bool TIMED, bool XP = false>
 __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -457,7 +484,9 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
     const unsigned long long g_start = timing ? global_timer_ns() : 0;
 
     // ---- shared-memory carve-up (mirrored by plan_launch on the host) --------------------------
-    const int xstride = p.G * p.K_L + 32;
+    // bytes of one token's row of staged X: int8, or packed (XP); the pad keeps the 8 tokens of an
+    // n-tile on different banks
+    const int xstride = XP ? p.G * p.K_L / 2 + 16 : p.G * p.K_L + 32;
     uint32_t* lut = reinterpret_cast<uint32_t*>(smem);                       // [256][lut_rep]
     uint32_t* lut1 = lut + 256 * p.lut_rep;                                  // [256] built first
     uint8_t* x8 = reinterpret_cast<uint8_t*>(lut1 + 256);
@@ -747,12 +776,18 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
                     int32_t sacc = 0;
                     uint4 vlo, vhi;
                     uint2 t;
-                    t = expand8(xpre[b].x, sacc); vlo.x = t.x; vlo.y = t.y;
-                    t = expand8(xpre[b].y, sacc); vlo.z = t.x; vlo.w = t.y;
-                    t = expand8(xpre[b].z, sacc); vhi.x = t.x; vhi.y = t.y;
-                    t = expand8(xpre[b].w, sacc); vhi.z = t.x; vhi.w = t.y;
-                    uint4* dst = reinterpret_cast<uint4*>(x8 + n * xstride + sgl * p.K_L + 32 * q);
-                    dst[0] = vlo; dst[1] = vhi;
+                    if (XP) {
+                        vlo.x = pack8(xpre[b].x, sacc); vlo.y = pack8(xpre[b].y, sacc);
+                        vlo.z = pack8(xpre[b].z, sacc); vlo.w = pack8(xpre[b].w, sacc);
+                        *reinterpret_cast<uint4*>(x8 + n * xstride + (sgl * p.K_L + 32 * q) / 2) = vlo;
+                    } else {
+                        t = expand8(xpre[b].x, sacc); vlo.x = t.x; vlo.y = t.y;
+                        t = expand8(xpre[b].y, sacc); vlo.z = t.x; vlo.w = t.y;
+                        t = expand8(xpre[b].z, sacc); vhi.x = t.x; vhi.y = t.y;
+                        t = expand8(xpre[b].w, sacc); vhi.z = t.x; vhi.w = t.y;
+                        uint4* dst = reinterpret_cast<uint4*>(x8 + n * xstride + sgl * p.K_L + 32 * q);
+                        dst[0] = vlo; dst[1] = vhi;
+                    }
                     if (x_upr == 32) {   // one warp holds exactly one (segment, token) pair
                         sacc = __reduce_add_sync(0xffffffffu, sacc);
                         if (lane == 0) sx16[pi] = sacc;
@@ -761,9 +796,9 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
                     }
                 }
             }
-            stage_x<NT>(p, kr * p.G, g_kr, x8, xstride, sx16, kXPre * (int)blockDim.x);
+            stage_x<NT, XP>(p, kr * p.G, g_kr, x8, xstride, sx16, kXPre * (int)blockDim.x);
         } else {
-            stage_x<NT>(p, kr * p.G, g_kr, x8, xstride, sx16, 0);
+            stage_x<NT, XP>(p, kr * p.G, g_kr, x8, xstride, sx16, 0);
         }
         __syncthreads();
     };
@@ -822,8 +857,9 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0;
             const uint32_t slot_a = smem_u32(my_ring + (size_t)cur * p.slot_bytes);
-            const uint32_t xb_a = smem_u32(x8) + (lane >> 2) * xstride + 8 * (lane & 3) + sgl * p.K_L;
-            process_tile<NT, 1>(slot_a, lut_a, 4u * (uint32_t)p.lut_rep, xb_a, xstride, p.mask_rows, lane, c);
+            const uint32_t xb_a = XP ? smem_u32(x8) + (lane >> 2) * xstride + 4 * (lane & 3) + sgl * (p.K_L / 2)
+                                     : smem_u32(x8) + (lane >> 2) * xstride + 8 * (lane & 3) + sgl * p.K_L;
+            process_tile<NT, 1, XP>(slot_a, lut_a, 4u * (uint32_t)p.lut_rep, xb_a, xstride, p.mask_rows, lane, c);
             __syncwarp();
             const long long t2c = timing ? clock64() : 0;
 
