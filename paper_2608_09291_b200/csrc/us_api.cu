@@ -185,17 +185,18 @@ void plan_classes(us_handle* h, int n_cta, std::vector<uint32_t> (&sched)[4])
         int sl = 0;
         const int G = local_plan(false, &sched[c], &sl);
         if (G > 0) { h->G[c] = G; h->s_local[c] = sl; }
-        // Packed X (N = 9..16 only: the kernel exists for that class) halves the shared memory of a
-        // K range at the price of three more integer instructions per n-tile and k-block. Worth it
-        // when it turns several K ranges into one (then no partial sum leaves the CTA).
+        // Packed X (N <= 16: the kernel exists for those classes) halves the shared memory of a K
+        // range at the price of three more integer instructions per n-tile and k-block. Worth it
+        // when it turns several K ranges into one (then no partial sum leaves the CTA; N = 8 on
+        // 5120 x 13824: 18.2 -> 15.1 us; where one range was enough already it costs 2-6 %).
         // Measured at N = 16: 28672 x 8192 38.4 -> 34.8 us and 4096 x 11008 17.9 -> 14.4 us (two
         // ranges become one); 5120 x 5120 12.0 -> 9.4 us (one range either way, but a CTA's share is
         // small and the staging pass and the freed shared memory count for more than the decode);
         // 13824 x 5120 15.7 -> 16.0 us (one range either way, long decode): not taken there.
-        if (nt == 2 && xp_knob() != 0) {
+        if (nt <= 2 && xp_knob() != 0) {
             const int64_t n_segs = h->host.n_segs;
             const int64_t ranges = (n_segs + h->G[c] - 1) / h->G[c];
-            const bool small_share = (int64_t)h->host.blob.size() / std::max(1, n_cta) < 128 * 1024;
+            const bool small_share = nt == 2 && (int64_t)h->host.blob.size() / std::max(1, n_cta) < 128 * 1024;
             if (ranges > 1 || small_share || xp_knob() == 2) {
                 std::vector<uint32_t> alt;
                 int sl2 = 0;
@@ -231,9 +232,11 @@ cudaError_t launch_st(const us::SpmmParams& p, bool xp, int grid, int block, int
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     const bool la = p.s_local > 0, timed = p.timers != nullptr;
-    if (NT == 2 && xp && la)   // packed X: planned for this class and local mode only
-        return timed ? cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<2, ST, true, true, true>, p)
-                     : cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<2, ST, true, false, true>, p);
+    if (NT <= 2 && xp && la) {   // packed X: planned for these classes and local mode only
+        constexpr int NP = NT <= 2 ? NT : 2;
+        return timed ? cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NP, ST, true, true, true>, p)
+                     : cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NP, ST, true, false, true>, p);
+    }
     if (la && !timed) return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, ST, true, false>, p);
     if (!la && !timed) return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, ST, false, false>, p);
     if (la) return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, ST, true, true>, p);
@@ -276,6 +279,10 @@ cudaError_t enable_large_smem(int bytes)
     if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<2, 2, true, false, true>, attr, bytes);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<2, 1, true, true, true>, attr, bytes);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<2, 2, true, true, true>, attr, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<1, 1, true, false, true>, attr, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<1, 2, true, false, true>, attr, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<1, 1, true, true, true>, attr, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<1, 2, true, true, true>, attr, bytes);
     return e;
 }
 

@@ -86,6 +86,16 @@ def test_layer_13b_shapes(b):
         _check_case(b, W, X, [16], s_w, s_x, max_N=16)
 
 
+def test_long_k_single_range_with_packed_activations(b):
+    """5120 x 13824 at 50 %: at N <= 8 the whole K extent fits one K range only with the
+    activations staged packed (the launch plan picks that); N = 16 needs two ranges."""
+    W = workloads.make_weight(5120, 13824, 0.5, seed=411)
+    X = workloads.make_x(13824, 16, seed=411)
+    s_w, s_x = workloads.make_scales(5120, 16, seed=411)
+    _check_case(b, W, X, [3, 8, 16], s_w, s_x, max_N=16)
+    _check_case(b, W, X, [8], max_N=8)
+
+
 @pytest.mark.parametrize("M,K,seed", [(28672, 8192, 500), (8192, 28672, 501)])
 def test_ffn_70b_full_size(b, M, K, seed):
     """Full-size 70B FFN shapes in the launch configuration the bench times: every output for
