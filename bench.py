@@ -520,16 +520,17 @@ def run_only(args):
     f = args.only.split(",")
     M, K, s, N = int(f[0]), int(f[1]), float(f[2]), int(f[3])
     fp16 = len(f) > 4 and f[4] == "fp16"
-    fmt = (16, int(f[5]), 2, 1) if len(f) > 5 else None
+    fmt = (16, int(f[5]), 2, 1) if len(f) > 5 and int(f[5]) > 0 else None
+    n_max = int(f[6]) if len(f) > 6 else N   # largest N the handles are encoded for
     torch.cuda.set_device(0)
     l2 = torch.cuda.get_device_properties(0).L2_cache_size or L2_BYTES_FALLBACK
     W = workloads.make_weight(M, K, s, seed=1)
-    X = workloads.make_x(K, N, seed=1)
-    s_w, s_x = workloads.make_scales(M, N, seed=1)
-    probe = binding.us_encode(W, None, fmt, N, binding.US_ENCODE_HOST_ONLY)
+    X = workloads.make_x(K, n_max, seed=1)
+    s_w, s_x = workloads.make_scales(M, n_max, seed=1)
+    probe = binding.us_encode(W, None, fmt, n_max, binding.US_ENCODE_HOST_ONLY)
     st = binding.us_get_stats(probe)
     binding.us_destroy(probe)
-    case = Case(binding, torch, W, s_w, X, s_x, N, replicas_for(st, l2), fmt=fmt)
+    case = Case(binding, torch, W, s_w, X, s_x, n_max, replicas_for(st, l2), fmt=fmt)
     for _ in range(max(1, args.warmup)):
         case.enqueue_pass(N, fp16)
     torch.cuda.synchronize()
@@ -571,7 +572,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-sweep", action="store_true")
-    ap.add_argument("--only", default=None, metavar="M,K,s,N[,int32|fp16[,K_L]]",
+    ap.add_argument("--only", default=None, metavar="M,K,s,N[,int32|fp16[,K_L[,N_max]]]",
                     help="time one case only (a few launches, no graph): the small run used for ncu captures")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
