@@ -185,7 +185,7 @@ void plan_classes(us_handle* h, int n_cta, std::vector<uint32_t> (&sched)[4])
         int sl = 0;
         const int G = local_plan(false, &sched[c], &sl);
         if (G > 0) { h->G[c] = G; h->s_local[c] = sl; }
-        // Packed X (N <= 16: the kernel exists for those classes) halves the shared memory of a K
+        // Packed X (N <= 32: the kernel exists for those classes) halves the shared memory of a K
         // range at the price of three more integer instructions per n-tile and k-block. Worth it
         // when it turns several K ranges into one (then no partial sum leaves the CTA; N = 8 on
         // 5120 x 13824: 18.2 -> 15.1 us; where one range was enough already it costs 2-6 %).
@@ -193,15 +193,19 @@ void plan_classes(us_handle* h, int n_cta, std::vector<uint32_t> (&sched)[4])
         // ranges become one); 5120 x 5120 12.0 -> 9.4 us (one range either way, but a CTA's share is
         // small and the staging pass and the freed shared memory count for more than the decode);
         // 13824 x 5120 15.7 -> 16.0 us (one range either way, long decode): not taken there.
-        if (nt <= 2 && xp_knob() != 0) {
+        if (nt <= 4 && xp_knob() != 0) {
             const int64_t n_segs = h->host.n_segs;
-            const int64_t ranges = (n_segs + h->G[c] - 1) / h->G[c];
+            const int64_t ranges = h->s_local[c] > 0 ? (n_segs + h->G[c] - 1) / h->G[c] : n_segs + 1;
             const bool small_share = nt == 2 && (int64_t)h->host.blob.size() / std::max(1, n_cta) < 128 * 1024;
             if (ranges > 1 || small_share || xp_knob() == 2) {
                 std::vector<uint32_t> alt;
                 int sl2 = 0;
                 const int G2 = local_plan(true, &alt, &sl2);
-                if (G2 > 0 && ((n_segs + G2 - 1) / G2 == 1 || xp_knob() == 2)) {
+                const int64_t ranges2 = G2 > 0 ? (n_segs + G2 - 1) / G2 : 0;
+                // (N = 32, packed against plain: 11008 x 4096 21.4 -> 18.5 us, 13824 x 5120 24.9 -> 23.6 us,
+                // 5120 x 5120 17.3 -> 18.2 us with one range; three ranges instead of eleven one-segment
+                // ranges on 4096 x 11008 were slower, 19.3 -> 26.4 us: only a single range pays)
+                if (G2 > 0 && (ranges2 == 1 || xp_knob() == 2)) {
                     h->G[c] = G2; h->s_local[c] = sl2; h->xp[c] = true;
                     sched[c] = alt;
                 }
@@ -232,8 +236,8 @@ cudaError_t launch_st(const us::SpmmParams& p, bool xp, int grid, int block, int
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     const bool la = p.s_local > 0, timed = p.timers != nullptr;
-    if (NT <= 2 && xp && la) {   // packed X: planned for these classes and local mode only
-        constexpr int NP = NT <= 2 ? NT : 2;
+    if (NT <= 4 && xp && la) {   // packed X: planned for these classes and local mode only
+        constexpr int NP = NT <= 4 ? NT : 4;
         return timed ? cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NP, ST, true, true, true>, p)
                      : cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NP, ST, true, false, true>, p);
     }
@@ -283,6 +287,10 @@ cudaError_t enable_large_smem(int bytes)
     if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<1, 2, true, false, true>, attr, bytes);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<1, 1, true, true, true>, attr, bytes);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<1, 2, true, true, true>, attr, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<4, 1, true, false, true>, attr, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<4, 2, true, false, true>, attr, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<4, 1, true, true, true>, attr, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<4, 2, true, true, true>, attr, bytes);
     return e;
 }
 
