@@ -693,7 +693,7 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
         spre.have_sx = true;
     }
     const int g_first = (kr_first == n_kr - 1) ? g_last : p.G;   // segments in that range
-    constexpr int kXPre = NT == 1 ? 8 : NT == 2 ? 4 : 0;   // 16-byte units of X a thread prefetches
+    constexpr int kXPre = NT <= 4 ? 8 : 0;   // 16-byte units of X a thread prefetches
     const int x_sh = 31 - __clz(p.K_L / 32);   // log2(units per (segment, token)) when a power of two
     const bool x_early = kXPre > 0 && p.x_fast == 2 && (1 << x_sh) == p.K_L / 32;
     uint4 xpre[kXPre > 0 ? kXPre : 1];
