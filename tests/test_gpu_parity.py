@@ -211,3 +211,30 @@ def test_back_to_back_launches_share_a_handle(b, M, K, N):
             assert (c == (ref2 if i % 2 == 0 else ref1)).all(), i
     finally:
         sw.close()
+
+
+def test_chain_of_different_matrices_without_synchronisation(b):
+    """Several encoded matrices of different shapes and launch plans (half-SM and full-SM CTAs,
+    one and several K ranges, int8 and packed activations) enqueued back to back on one stream,
+    many rounds, no synchronisation in between: consecutive launches of different kernels overlap
+    their prologues, and each must still see exactly its own inputs, workspace and output."""
+    shapes = [(1024, 1024, 8), (4096, 2048, 8), (2048, 4096, 16), (5120, 1024, 8), (768, 8192, 16),
+              (3072, 3072, 32), (2048, 12288, 8)]
+    cases = []
+    try:
+        for i, (M, K, N) in enumerate(shapes):
+            W = workloads.make_weight(M, K, (0.5, 0.3, 0.7)[i % 3], seed=900 + i)
+            X = workloads.make_x(K, N, seed=900 + i)
+            sw = b.SparseWeight(W, None, max_N=N)
+            cases.append((sw, W, X, N, torch.from_numpy(b.pack_int4(X)).cuda(),
+                          torch.zeros((N, M), dtype=torch.int32, device="cuda")))
+        for rnd in range(15):
+            for sw, W, X, N, Xd, Y in (cases if rnd % 2 == 0 else cases[::-1]):
+                sw.spmm(Xd, N, out=Y)
+        torch.cuda.synchronize()
+        for sw, W, X, N, Xd, Y in cases:
+            sw.check()
+            assert (Y.cpu().numpy() == oracle.spmm_dense(W, X)).all(), (W.shape, N)
+    finally:
+        for c in cases:
+            c[0].close()
