@@ -169,7 +169,7 @@ def dequant(acc: np.ndarray, s_w: np.ndarray, s_x: np.ndarray) -> np.ndarray:
 
 def fp16_within_tolerance(got: np.ndarray, ref_acc: np.ndarray, s_w: np.ndarray,
                           s_x: np.ndarray, rel: float = 2e-3) -> np.ndarray:
-    """Element-wise verdict of the stated bar: |got - exact| <= max(rel*|exact|, 1 fp16 ulp of
+    """Element-wise check against the stated bar: |got - exact| <= max(rel*|exact|, 1 fp16 ulp of
     the correctly rounded reference)."""
     sw = np.asarray(s_w, dtype=np.float16).astype(np.float64)
     sx = np.asarray(s_x, dtype=np.float16).astype(np.float64)
