@@ -17,6 +17,7 @@ struct us_handle {
     int max_N = 0;
     int max_smem = 0;
     int co_warps = 10;   // warps of an N <= 8 CTA when two CTAs share an SM's registers
+    int co_warps2 = 8;   // the same for the N = 9..16 kernel with packed activations
     uint8_t* d_blob = nullptr;
     uint32_t* d_item_off = nullptr;
     std::vector<uint32_t> cta_begin[4];  // schedule per N class (NT = 1, 2, 4, 8)
@@ -141,10 +142,12 @@ bool plan_launch(const us_handle* h, int N, LaunchGeom* g)
     // Measured on 4096 x 4096, N = 8: 6.6 -> 5.7 us; not worth it from ~20 tiles per CTA on.
     const int64_t per_cta = (h->host.n_items + 147) / 148;
     int fixed = fixed_base + 32 * stages * 8;
-    if (coresident_knob() && g->nt == 1 && per_cta <= 16 && stages_knob() == 0 && lut_rep_knob() == 0) {
+    // (N = 9..16 too, where the plan stages X packed and in local mode: that kernel is as lean.)
+    const bool co_class = g->nt == 1 || (g->nt == 2 && g->xp && s_local > 0);
+    if (coresident_knob() && co_class && per_cta <= 16 && stages_knob() == 0 && lut_rep_knob() == 0) {
         const int half = 228 * 1024 / 2 - 1024 - 512;   // per SM: 228 KB, 1 KB reserved per CTA
         const int fixed8 = fixed_for(8) + 32 * 8;
-        int w = std::min(h->co_warps, max_warps());
+        int w = std::min(g->nt == 1 ? h->co_warps : h->co_warps2, max_warps());
         while (w >= 8 && fixed8 + w * (int)g->slot_bytes > half) --w;
         if (w >= 8) { stages = 1; lut_rep = 8; warps = w; fixed = fixed8; }
     }
@@ -357,6 +360,9 @@ us_status us_encode(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_sca
             regs = std::max(regs, fa.numRegs);
         }
         if (e == cudaSuccess) h->co_warps = 32768 / (32 * ((regs + 7) / 8 * 8));
+        cudaFuncAttributes fa2;
+        if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa2, (const void*)us::us_spmm_kernel<2, 1, true, false, true>);
+        if (e == cudaSuccess) h->co_warps2 = 32768 / (32 * ((fa2.numRegs + 7) / 8 * 8));
     }
     if (e != cudaSuccess) { delete h; return US_ERR_CUDA; }
 
