@@ -143,6 +143,7 @@ bool plan_launch(const us_handle* h, int N, LaunchGeom* g)
     const int64_t per_cta = (h->host.n_items + 147) / 148;
     int fixed = fixed_base + 32 * stages * 8;
     // (N = 9..16 too, where the plan stages X packed and in local mode: that kernel is as lean.)
+    // (Tried at N = 32 as well: 8 warps per CTA, slower.)
     const bool co_class = g->nt == 1 || (g->nt == 2 && g->xp && s_local > 0);
     if (coresident_knob() && co_class && per_cta <= 16 && stages_knob() == 0 && lut_rep_knob() == 0) {
         const int half = 228 * 1024 / 2 - 1024 - 512;   // per SM: 228 KB, 1 KB reserved per CTA
@@ -199,7 +200,7 @@ void plan_classes(us_handle* h, int n_cta, std::vector<uint32_t> (&sched)[4])
         if (nt <= 4 && xp_knob() != 0) {
             const int64_t n_segs = h->host.n_segs;
             const int64_t ranges = h->s_local[c] > 0 ? (n_segs + h->G[c] - 1) / h->G[c] : n_segs + 1;
-            const bool small_share = nt == 2 && (int64_t)h->host.blob.size() / std::max(1, n_cta) < 128 * 1024;
+            const bool small_share = nt >= 2 && (int64_t)h->host.blob.size() / std::max(1, n_cta) < 128 * 1024;
             if (ranges > 1 || small_share || xp_knob() == 2) {
                 std::vector<uint32_t> alt;
                 int sl2 = 0;
@@ -363,6 +364,7 @@ us_status us_encode(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_sca
         cudaFuncAttributes fa2;
         if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa2, (const void*)us::us_spmm_kernel<2, 1, true, false, true>);
         if (e == cudaSuccess) h->co_warps2 = 32768 / (32 * ((fa2.numRegs + 7) / 8 * 8));
+
     }
     if (e != cudaSuccess) { delete h; return US_ERR_CUDA; }
 
