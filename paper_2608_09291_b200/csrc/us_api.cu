@@ -52,6 +52,7 @@ int local_acc_budget() { static int v = env_int("US_LOCAL_ACC_KB", 32) * 1024; r
 int stages_knob() { static int v = env_int("US_STAGES", 0); return v; }     // ring slots per warp, 0 = automatic
 int lut_rep_knob() { static int v = env_int("US_LUT_REP", 0); return v; }   // selector-table copies, 0 = automatic
 int pdl_knob() { static int v = env_int("US_PDL", 1); return v; }          // programmatic dependent launch
+int coresident_tiles_knob() { static int v = env_int("US_CORESIDENT_TILES", 16); return v; }
 int coresident_knob() { static int v = env_int("US_CORESIDENT", 1); return v; }  // small problems: half an SM per CTA
 int max_warps() { static int v = std::min(16, std::max(2, env_int("US_MAX_WARPS", 16))); return v; }
 
@@ -145,7 +146,7 @@ bool plan_launch(const us_handle* h, int N, LaunchGeom* g)
     // (N = 9..16 too, where the plan stages X packed and in local mode: that kernel is as lean.)
     // (Tried at N = 32 as well: 8 warps per CTA, slower.)
     const bool co_class = g->nt == 1 || (g->nt == 2 && g->xp && s_local > 0);
-    if (coresident_knob() && co_class && per_cta <= 16 && stages_knob() == 0 && lut_rep_knob() == 0) {
+    if (coresident_knob() && co_class && per_cta <= coresident_tiles_knob() && stages_knob() == 0 && lut_rep_knob() == 0) {
         const int half = 228 * 1024 / 2 - 1024 - 512;   // per SM: 228 KB, 1 KB reserved per CTA
         const int fixed8 = fixed_for(8) + 32 * 8;
         int w = std::min(g->nt == 1 ? h->co_warps : h->co_warps2, max_warps());
