@@ -3,6 +3,7 @@
 #include <algorithm>
 #include <climits>
 #include <atomic>
+#include <cstdlib>
 #include <cstring>
 #include <numeric>
 #include <thread>
@@ -305,18 +306,23 @@ void make_schedule(const HostMatrix& h, int n_cta, int G, std::vector<uint32_t>*
             }
     }
     const uint64_t total = prefix[h.n_items];
-    // Small matrices (a CTA's share is only a few strips, all in one K range): cut at strip
-    // boundaries. A strip then lives in one CTA and is stored straight from shared memory; the
-    // global reduce (fence, counter, re-read) would cost more than the coarser balance loses.
-    const bool whole_strips = (n_kr == 1) && (h.n_strips < (int64_t)4 * n_cta);
+    // Cuts fall on strip boundaries (within their K range): every strip's tiles of a range are then
+    // summed inside one CTA. With one K range nothing goes through the global split-K workspace at
+    // all; that is worth far more than the finer byte balance of cutting inside strips (measured at
+    // N = 8: 11008 x 4096 11.2 -> 9.0 us, 13824 x 5120 13.4 -> 11.2 us, 28672 x 8192 26.6 -> 25.0 us).
+    static const int align_mode = [] { const char* e = std::getenv("US_STRIP_CUTS"); return e ? std::atoi(e) : 2; }();
+    // 0: only small matrices in one K range (< 4 strips per CTA); 1: always with one K range; 2: always
+    const bool whole_strips = align_mode >= 2 || (n_kr == 1 && (align_mode == 1 || h.n_strips < (int64_t)4 * n_cta));
+    const int64_t g_last = h.n_segs - (n_kr - 1) * G;
     int64_t pos = 0;
     for (int c = 0; c <= n_cta; ++c) {
         const uint64_t target = total * (uint64_t)c / (uint64_t)n_cta;
         while (pos < h.n_items && prefix[pos] < target) ++pos;
         if (whole_strips && pos < h.n_items) {
-            // round to the nearest strip boundary (in bytes)
-            const int64_t g = h.n_segs;
-            const int64_t down = pos / g * g, up = std::min<int64_t>(h.n_items, down + g);
+            // round to the nearest strip boundary of the position's K range (in bytes)
+            const int64_t kr = kr_of[pos];
+            const int64_t base = kr * h.n_strips * G, g = (kr == n_kr - 1) ? g_last : G;
+            const int64_t down = base + (pos - base) / g * g, up = std::min<int64_t>(h.n_items, down + g);
             pos = (prefix[pos] - prefix[down] <= prefix[up] - prefix[pos]) ? down : up;
         }
         (*begin)[c] = (uint32_t)std::max<int64_t>(pos, c ? (int64_t)(*begin)[c - 1] : 0);
