@@ -306,11 +306,12 @@ void make_schedule(const HostMatrix& h, int n_cta, int G, std::vector<uint32_t>*
             }
     }
     const uint64_t total = prefix[h.n_items];
-    // Cuts fall on strip boundaries (within their K range): every strip's tiles of a range are then
-    // summed inside one CTA. With one K range nothing goes through the global split-K workspace at
-    // all; that is worth far more than the finer byte balance of cutting inside strips (measured at
-    // N = 8: 11008 x 4096 11.2 -> 9.0 us, 13824 x 5120 13.4 -> 11.2 us, 28672 x 8192 26.6 -> 25.0 us).
-    static const int align_mode = [] { const char* e = std::getenv("US_STRIP_CUTS"); return e ? std::atoi(e) : 2; }();
+    // With one K range the cuts fall on strip boundaries: every strip is then summed inside one CTA
+    // and nothing goes through the global split-K workspace at all; that is worth far more than the
+    // finer byte balance of cutting inside strips (measured at N = 8: 11008 x 4096 11.2 -> 9.0 us,
+    // 13824 x 5120 13.4 -> 11.2 us, 28672 x 8192 26.6 -> 25.0 us). With several K ranges every strip
+    // goes through the workspace anyway and aligned cuts make no measurable difference.
+    static const int align_mode = [] { const char* e = std::getenv("US_STRIP_CUTS"); return e ? std::atoi(e) : 1; }();
     // 0: only small matrices in one K range (< 4 strips per CTA); 1: always with one K range; 2: always
     const bool whole_strips = align_mode >= 2 || (n_kr == 1 && (align_mode == 1 || h.n_strips < (int64_t)4 * n_cta));
     const int64_t g_last = h.n_segs - (n_kr - 1) * G;
