@@ -323,7 +323,8 @@ void make_schedule(const HostMatrix& h, int n_cta, int G, std::vector<uint32_t>*
     // costs 2 %.
     static const int tilt = [] { const char* e = std::getenv("US_TILT"); return e ? std::atoi(e) : 30; }();
     for (int c = 0; c <= n_cta; ++c) {
-        const double x = (double)c / (double)n_cta, a = tilt * 1e-3;
+        // (only where a CTA's share is many strips: on small shares the rounding to strips decides)
+        const double x = (double)c / (double)n_cta, a = (whole_strips && h.n_strips >= (int64_t)8 * n_cta) ? tilt * 1e-3 : 0.0;
         const uint64_t target = (uint64_t)((double)total * (x + a * x * (1.0 - x)));
         while (pos < h.n_items && prefix[pos] < target) ++pos;
         if (whole_strips && pos < h.n_items) {
