@@ -337,6 +337,41 @@ void make_schedule(const HostMatrix& h, int n_cta, int G, std::vector<uint32_t>*
         (*begin)[c] = (uint32_t)std::max<int64_t>(pos, c ? (int64_t)(*begin)[c - 1] : 0);
     }
     (*begin)[n_cta] = (uint32_t)h.n_items;
+    // Several K ranges: no CTA should straddle a range boundary -- changing range costs a CTA a full
+    // restaging of X behind a CTA-wide barrier (about 9 K cycles), and the whole launch waits for
+    // those few CTAs. Give every range a whole number of CTAs in proportion to its bytes and split
+    // each range evenly among its own.
+    static const int range_mode = [] { const char* e = std::getenv("US_RANGE_CTAS"); return e ? std::atoi(e) : 1; }();
+    // (Not with one-segment ranges -- the direct mode: there a range is small, changing it is cheap,
+    // and rounding CTAs to many ranges unbalances them: N = 64 on 28672 x 8192 87 -> 93 us.)
+    if (range_mode && n_kr > 1 && G > 1 && n_kr * 8 <= n_cta) {
+        std::vector<int64_t> r_beg((size_t)n_kr + 1, 0);
+        for (int64_t kr = 0; kr < n_kr; ++kr) r_beg[kr + 1] = std::min<int64_t>(h.n_items, (kr + 1) * h.n_strips * G);
+        r_beg[n_kr] = h.n_items;
+        std::vector<int> n_of((size_t)n_kr, 1);
+        int used = (int)n_kr;
+        std::vector<double> want((size_t)n_kr);
+        for (int64_t kr = 0; kr < n_kr; ++kr)
+            want[kr] = (double)(prefix[r_beg[kr + 1]] - prefix[r_beg[kr]]) / (double)std::max<uint64_t>(1, total) * n_cta;
+        while (used < n_cta) {   // one more CTA to the range that is furthest below its fair number
+            int64_t best = 0;
+            for (int64_t kr = 1; kr < n_kr; ++kr)
+                if (want[kr] - n_of[kr] > want[best] - n_of[best]) best = kr;
+            ++n_of[best];
+            ++used;
+        }
+        int c = 0;
+        for (int64_t kr = 0; kr < n_kr; ++kr) {
+            const uint64_t b0 = prefix[r_beg[kr]], b1 = prefix[r_beg[kr + 1]];
+            int64_t q = r_beg[kr];
+            for (int i = 0; i < n_of[kr]; ++i, ++c) {
+                const uint64_t target = b0 + (b1 - b0) * (uint64_t)i / (uint64_t)n_of[kr];
+                while (q < r_beg[kr + 1] && prefix[q] < target) ++q;
+                (*begin)[c] = (uint32_t)q;
+            }
+        }
+        (*begin)[n_cta] = (uint32_t)h.n_items;
+    }
     int worst = 1;
     for (int c = 0; c < n_cta; ++c) {
         int64_t a = (*begin)[c], b = (*begin)[c + 1];
