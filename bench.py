@@ -423,6 +423,7 @@ def sweep(binding, torch, workloads, l2, peak_gbs):
     run_case("attn7b_qkv_fused", 12288, 4096, 0.5, 210, [8], True)   # Q, K, V stacked: one launch
     run_case("ffn7b_up", 11008, 4096, 0.5, 300, [8], True, row_varying=True, flags=binding.US_ENCODE_SORT_ROWS)
     run_case("ffn70b_up", 28672, 8192, 0.6, 500, [1, 4, 8, 16, 32, 64], False)
+    run_case("ffn70b_down", 8192, 28672, 0.6, 501, [1, 4, 8, 16, 32, 64], False)
     # Bitmap-aware row pairing inside each strip (the per-strip form of Alg. 1): fewer union bits.
     run_case("attn7b_paired", 4096, 4096, 0.5, 201, [8], True, flags=binding.US_ENCODE_PAIR_ROWS)
     run_case("ffn70b_up_paired", 28672, 8192, 0.6, 500, [8], False, flags=binding.US_ENCODE_PAIR_ROWS)
