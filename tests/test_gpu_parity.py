@@ -238,3 +238,23 @@ def test_chain_of_different_matrices_without_synchronisation(b):
     finally:
         for c in cases:
             c[0].close()
+
+
+def test_seeded_random_shapes(b):
+    """Forty seeded random problems -- shape, sparsity, N, tile width, row-order flags -- each
+    checked element by element (INT32 exact, fp16 within the bar), twice per handle."""
+    rng = np.random.default_rng(20240917)
+    for case in range(40):
+        M = int(rng.integers(1, 700))
+        K = int(rng.integers(1, 6000))
+        s = float(rng.choice([0.0, 0.3, 0.5, 0.7, 0.9, 1.0]))
+        N = int(rng.integers(1, 65))
+        K_L = int(rng.choice([128, 256, 512, 1024]))
+        flags = int(rng.choice([0, 2, 4, 6]))
+        W = workloads.make_weight(M, K, s, seed=7000 + case, row_varying=bool(flags & 2))
+        X = workloads.make_x(K, N, seed=7000 + case)
+        s_w, s_x = workloads.make_scales(M, N, seed=7000 + case)
+        try:
+            _check_case(b, W, X, [N], s_w, s_x, fmt=(16, K_L, 2, 1), flags=flags, max_N=N)
+        except AssertionError as e:
+            raise AssertionError(f"case {case}: M={M} K={K} s={s} N={N} K_L={K_L} flags={flags}: {e}")
