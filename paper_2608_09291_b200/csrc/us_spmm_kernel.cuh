@@ -738,13 +738,18 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
     };
     // announce n_tiles finished contributions to strip rb; the arrival that completes it finalizes
     auto signal_strip = [&](int rb, uint32_t n_tiles, int m_lo, int m_hi) {
-        __threadfence();
+        // One acquire-release add instead of fence + add + fence: the warp barrier orders every
+        // lane's adds to the workspace before lane 0's release; the arrival that completes the strip
+        // acquires every earlier contributor's adds, and the second warp barrier hands that to the
+        // other lanes. (Measured against the three-step form: N = 32 on 28672 x 8192 52.8 -> 48.8 us,
+        // N = 8 on 8192 x 28672 28.7 -> 27.6 us.)
         __syncwarp();
         uint32_t old = 0;
-        if (lane == 0) old = atomicAdd(p.cnt + rb, n_tiles);
+        if (lane == 0)
+            asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(old) : "l"(p.cnt + rb), "r"(n_tiles) : "memory");
         old = __shfl_sync(0xffffffffu, old, 0);
         if (old + n_tiles == (uint32_t)p.n_segs) {
-            __threadfence();
+            __syncwarp();
             if (m_lo == kNoRow) {
                 m_lo = __ldg(p.row_order + rb * 16 + (lane >> 2));
                 m_hi = __ldg(p.row_order + rb * 16 + (lane >> 2) + 8);
