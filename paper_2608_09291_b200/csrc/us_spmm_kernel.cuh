@@ -919,13 +919,16 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
                         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
                             for (int j = 0; j < 4; ++j) atomicAdd(al + nt * 128 + j * 32, y[nt][j]);
-                        __threadfence_block();
+                        // (one acquire-release add on the strip's counter instead of fence, add, fence:
+                        // as for the global workspace below, with the warp barriers on both sides)
                         __syncwarp();
                         uint32_t old = 0;
-                        if (lane == 0) old = atomicAdd(cnt_l + (rb - rb_first), y_n);
+                        if (lane == 0)
+                            asm volatile("atom.acq_rel.cta.shared.add.u32 %0, [%1], %2;"
+                                         : "=r"(old) : "r"(smem_u32(cnt_l + (rb - rb_first))), "r"(y_n) : "memory");
                         old = __shfl_sync(0xffffffffu, old, 0);
                         if (old + y_n == expected) {   // the CTA's last tiles of this strip: flush it
-                            __threadfence_block();
+                            __syncwarp();
 #pragma unroll
                             for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
