@@ -115,7 +115,7 @@ def reference_arm(args, rank: int):
     W = workloads.make_weight(HEAD["M"], HEAD["K"], HEAD["s"], HEAD["seed"])
     X = workloads.make_x(HEAD["K"], 32, HEAD["seed"])[: HEAD["N"]]
     s_w, s_x = workloads.make_scales(HEAD["M"], 32, HEAD["seed"])
-    st = oracle.encode(W, 16, 1024, 2, 1)["stats"]
+    st = oracle.encode(W, 16, 512, 2, 1)["stats"]
     stats = dict(M=HEAD["M"], K=HEAD["K"], bytes_payload=st["bytes_payload"],
                  bytes_bitmap=st["bytes_bitmap"], bytes_offsets=st["bytes_offsets"])
     per_call = algorithmic_bytes(stats, HEAD["N"], True)
