@@ -53,6 +53,7 @@ int stages_knob() { static int v = env_int("US_STAGES", 0); return v; }     // r
 int lut_rep_knob() { static int v = env_int("US_LUT_REP", 0); return v; }   // selector-table copies, 0 = automatic
 int pdl_knob() { static int v = env_int("US_PDL", 1); return v; }          // programmatic dependent launch
 int coresident_tiles_knob() { static int v = env_int("US_CORESIDENT_TILES", 16); return v; }
+int local_acc_cap() { static int v = env_int("US_LOCAL_ACC_CAP_KB", 48) * 1024; return v; }
 int coresident_knob() { static int v = env_int("US_CORESIDENT", 1); return v; }  // small problems: half an SM per CTA
 int max_warps() { static int v = std::min(16, std::max(2, env_int("US_MAX_WARPS", 16))); return v; }
 
@@ -171,16 +172,29 @@ void plan_classes(us_handle* h, int n_cta, std::vector<uint32_t> (&sched)[4])
         // last range spreads a CTA over more strips, so shorter ranges are tried before giving up.
         // Returns the range length found (0 = none) and leaves the schedule in `out`.
         auto local_plan = [&](bool xp, std::vector<uint32_t>* out, int* s_local) -> int {
-            int G = 0, worst = 1;
-            for (int64_t r = 1; r <= h->host.n_segs; ++r) {
-                const int Gr = segs_per_range(h->host, nt, limit, r, xp);
-                if (Gr == G) continue;
-                G = Gr;
-                if (G <= 1) break;
-                us::make_schedule(h->host, n_cta, G, out, &worst);
-                if (plan_debug())
-                    fprintf(stderr, "[unionsparse] plan nt=%d%s: G=%d needs %d local strips\n", nt, xp ? " packed X" : "", G, worst);
-                if (worst * nt * 512 <= local_acc_budget()) { *s_local = worst; return G; }
+            // second pass: a little more than the budget the range length was chosen with is taken
+            // if nothing fits the budget and at least 11 warps remain -- the alternative is the global
+            // split-K path for every tile (N = 32: 5120 x 13824 30.2 -> 22.4 us, 4096 x 11008 18.7 ->
+            // 16.2 us; N = 64 on 5120 x 5120 25.3 -> 19.5 us)
+            for (int pass = 0; pass < 2; ++pass) {
+                int G = 0, worst = 1;
+                for (int64_t r = 1; r <= h->host.n_segs; ++r) {
+                    const int Gr = segs_per_range(h->host, nt, limit, r, xp);
+                    if (Gr == G) continue;
+                    G = Gr;
+                    if (G <= 1) break;
+                    us::make_schedule(h->host, n_cta, G, out, &worst);
+                    const int need = worst * nt * 512;
+                    if (plan_debug())
+                        fprintf(stderr, "[unionsparse] plan nt=%d%s: G=%d needs %d local strips\n", nt, xp ? " packed X" : "", G, worst);
+                    if (pass == 0 && need <= local_acc_budget()) { *s_local = worst; return G; }
+                    if (pass == 1 && need <= local_acc_cap()) {
+                        const int slot = (int)((h->host.max_item_bytes + 256u + 127u) & ~127u);
+                        const int64_t fixed = 256 * 8 * 4 + (int64_t)us::kLutScratchBytes + need + 2 * us::kOffTable * 4 + 1024 +
+                                              x_bytes(nt, G, h->host.fmt.K_L, xp) + (int64_t)G * nt * 32;
+                        if ((limit - fixed) / slot >= 11) { *s_local = worst; return G; }
+                    }
+                }
             }
             return 0;
         };
