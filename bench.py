@@ -447,7 +447,9 @@ def sweep(binding, torch, workloads, l2, peak_gbs):
     for i, s in enumerate((0.3, 0.5, 0.7)):
         run_case("attn7b", 4096, 4096, s, 200 + i, [1, 8, 16, 32], True)
     run_case("attn7b_qkv_fused", 12288, 4096, 0.5, 210, [8], True)   # Q, K, V stacked: one launch
-    run_case("ffn7b_up", 11008, 4096, 0.5, 300, [8], True, row_varying=True, flags=binding.US_ENCODE_SORT_ROWS)
+    run_case("ffn7b_up", 11008, 4096, 0.5, 300, [1, 8, 32], True, row_varying=True, flags=binding.US_ENCODE_SORT_ROWS)
+    run_case("ffn7b_up", 11008, 4096, 0.5, 300, [8], False, row_varying=True, flags=binding.US_ENCODE_SORT_ROWS)
+    run_case("ffn7b_down", 4096, 11008, 0.5, 302, [1, 8, 32], True, row_varying=True, flags=binding.US_ENCODE_SORT_ROWS)
     run_case("ffn70b_up", 28672, 8192, 0.6, 500, [1, 4, 8, 16, 32, 64], False)
     run_case("ffn70b_down", 8192, 28672, 0.6, 501, [1, 4, 8, 16, 32, 64], False)
     # Bitmap-aware row pairing inside each strip (the per-strip form of Alg. 1): fewer union bits.

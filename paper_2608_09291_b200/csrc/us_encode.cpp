@@ -292,6 +292,17 @@ void make_schedule(const HostMatrix& h, int n_cta, int G, std::vector<uint32_t>*
     // segment within the range. Position u of that order maps to tile rb * n_segs + kr * G + sgl.
     begin->assign((size_t)n_cta + 1, 0);
     const int64_t n_kr = (h.n_segs + G - 1) / G;
+    // Cost of a tile in the balance: its bytes (units of 16) plus a constant. The decode works per
+    // k-block, whatever the payload: a tile of a sparse strip takes nearly as long as one of a dense
+    // strip, so balancing bytes alone overloads the CTAs that get the sparse strips. Measured on a
+    // row-varying 4096 x 11008 matrix with sorted rows: N = 8 11.5 -> 10.0 us, N = 32 25.5 -> 20.3 us
+    // with cost = bytes + 2 x the average tile; uniform matrices are unaffected.
+    // (US_BALANCE: 0 = bytes only, 1 = tiles only, k >= 2 = bytes + k x average tile)
+    static const int mode = [] { const char* e = std::getenv("US_BALANCE"); return e ? std::atoi(e) : 2; }();
+    const uint64_t avg16 = std::max<uint64_t>(1, h.item_off[h.n_items] / (uint64_t)std::max<int64_t>(1, h.n_items));
+    auto tile_cost = [&](uint32_t units16) -> uint64_t {
+        return mode == 0 ? units16 : mode == 1 ? avg16 : units16 + (uint64_t)mode * avg16;
+    };
     std::vector<uint64_t> prefix((size_t)h.n_items + 1, 0);
     std::vector<int32_t> strip_of((size_t)h.n_items), kr_of((size_t)h.n_items);
     int64_t u = 0;
@@ -300,7 +311,7 @@ void make_schedule(const HostMatrix& h, int n_cta, int G, std::vector<uint32_t>*
         for (int64_t rb = 0; rb < h.n_strips; ++rb)
             for (int64_t sgl = 0; sgl < g_kr; ++sgl, ++u) {
                 const int64_t t = rb * h.n_segs + kr * G + sgl;
-                prefix[u + 1] = prefix[u] + (h.item_off[t + 1] - h.item_off[t]);
+                prefix[u + 1] = prefix[u] + tile_cost(h.item_off[t + 1] - h.item_off[t]);
                 strip_of[u] = (int32_t)rb;
                 kr_of[u] = (int32_t)kr;
             }
