@@ -574,17 +574,25 @@ def run_only(args):
     t = e0.elapsed_time(e1) * 1e-3 / (args.steps * len(case.sw))
     alg = algorithmic_bytes(case.stats, N, fp16)
     t_graph = case.time_passes(N, fp16, passes=max(3, args.steps), warmup=3)
-    # one more pass with the kernel's stage timers on (not part of the timing above)
-    for sw in case.sw:
-        binding.us_stage_timers(sw.handle, 1)
+    # one more pass with the stage timers of ONE handle in the middle of the pass on (not part of
+    # the timing above): a single launch in the steady state of back-to-back launches
+    probe = case.sw[len(case.sw) // 2]
+    binding.us_stage_timers(probe.handle, 1)
     case.enqueue_pass(N, fp16)
     torch.cuda.synchronize()
-    tm = {}
-    for sw in case.sw:
-        for k, v in binding.us_stage_timers(sw.handle, 0, read=True).items():
-            tm[k] = tm.get(k, 0) + v
-    per_warp = ("wait", "decode", "epilogue", "lifetime", "prologue")
-    timers = {k: (v / max(1, tm["warps"]) if k in per_warp else v / len(case.sw)) for k, v in tm.items()}
+    d = binding.us_stage_timers(probe.handle, 0, read=True, per_cta=192)
+    ctas = [c for c in d.pop("ctas") if c[3]]
+    ck = d.pop("checkpoints")
+    timers = {k: (v / max(1, d["warps"]) if k in ("wait", "decode", "epilogue", "lifetime", "prologue") else v)
+              for k, v in d.items()}
+    timers["checkpoints"] = [v / max(1, d["warps"]) for v in ck]
+    if ctas:
+        t0 = min(c[0] for c in ctas)
+        q = lambda xs: [int(np.percentile(xs, pc)) for pc in (0, 50, 100)]
+        timers["cta_ns_min_med_max"] = {"start": q([c[0] - t0 for c in ctas]), "past_wait": q([c[4] - t0 for c in ctas]),
+                                        "x_stage": q([c[2] - c[4] for c in ctas]), "tail": q([c[3] - c[1] for c in ctas]),
+                                        "x_staged": q([c[2] - t0 for c in ctas]), "end": q([c[3] - t0 for c in ctas]),
+                                        "loop": q([c[3] - c[2] for c in ctas])}
     print(json.dumps({"only": args.only, "us_per_launch_graph": t_graph * 1e6, "gbs_graph": alg / t_graph / 1e9,
                       "us_per_launch_stream_order": t * 1e6, "alg_bytes": alg,
                       "stored_bytes": binding.us_spmm_bytes(case.sw[0].handle, N, fp16),

@@ -35,8 +35,12 @@ typedef enum us_status {
 /*
  * IE-BME format parameters (paper Sec. V-A "Area Partitioning"): a local tile of H_L x K_L
  * weights is split into an R_A x C_A grid of areas; one union-mask bit covers the Q = R_A*C_A
- * values at the same position of every area. Supported by the kernels: H_L = 16, K_L a multiple
- * of 128 (default 1024), (R_A, C_A) = (2, 1): one bit covers rows i and i+8 of a 16-row strip.
+ * values at the same position of every area. Every format whose union mask fills whole 64-bit
+ * words (the paper's {16, 64, 2, 2} among them, and per-element bitmaps {16, 64, 1, 1}) can be
+ * encoded, decoded and measured (us_get_stats) on a US_ENCODE_HOST_ONLY handle, in the paper's
+ * own array layout. The kernels implement H_L = 16, (R_A, C_A) = (2, 1) -- one bit covers rows i
+ * and i+8 of a 16-row strip -- with K_L a multiple of 128 up to 8192; only such handles can be
+ * uploaded and multiplied.
  */
 typedef struct us_format {
     int32_t H_L, K_L, R_A, C_A;
@@ -50,7 +54,8 @@ typedef struct us_stats {
     int64_t n_tiles;              /* local tiles (one offset each)                          */
     int64_t sum_P;                /* sum over tiles of P_t = active union-mask bits         */
     int64_t bytes_payload;        /* ceil(Q * sum_P / 2): the packed INT4 values            */
-    int64_t bytes_payload_padded; /* payload bytes as stored (lane streams padded per tile) */
+    int64_t bytes_payload_padded; /* payload bytes as stored (kernel layout: lane streams padded
+                                     per tile; the paper's layout stores no padding)        */
     int64_t bytes_bitmap;         /* union bitmaps                                          */
     int64_t bytes_offsets;        /* 4 * (n_tiles + 1)                                      */
     int64_t bytes_total;          /* bytes_payload_padded + bytes_bitmap + bytes_offsets    */
@@ -82,7 +87,8 @@ typedef struct us_handle us_handle;
  *   W        host, M x K row-major int8, values in [-8, 7], 0 = pruned. Not retained.
  *   w_scale  host, M fp16 bit patterns (per-output-channel scales), or NULL when only INT32
  *            output will be requested. Not retained.
- *   fmt      NULL selects {16, 1024, 2, 1}.
+ *   fmt      NULL selects {16, K_L, 2, 1} with K_L = 1024, 512 or 256 by the shape (long tiles
+ *            for large matrices, short ones where every SM must still find work).
  *   max_N    largest N later passed to us_spmm (1..64); sizes the split-K workspace.
  *   out      receives the handle; it owns every host and device array it allocates.
  * M, K need not be multiples of the tile: the matrix is zero padded internally.
@@ -118,7 +124,10 @@ us_status us_get_row_order(const us_handle* h, int32_t* perm_out);
  * Caller owns X, x_scale and Y. Returns before the kernel completes; device-side failures are
  * reported by us_last_error. One call per handle may be in flight: the split-K workspace and
  * arrival counters belong to the handle and are left zeroed by each call.
- * Errors: INVALID_ARG, UNSUPPORTED (host-only handle), CUDA.
+ * The handle's device must be the current device. After a call that us_last_error reports as
+ * failed, the workspace has been cleared again and the handle can be used as before.
+ * Errors: INVALID_ARG (also: another device is current), UNSUPPORTED (host-only handle, or a
+ * format no kernel reads), CUDA.
  */
 us_status us_spmm(us_handle* h, const void* X, int32_t N, const void* x_scale, void* Y,
                   void* stream);
@@ -154,21 +163,36 @@ us_status us_spmm_static_scratch(us_handle* h, const void* X, int32_t N, const v
 /*
  * Synchronises the device, then reports the first failure recorded for this handle: a CUDA
  * error of an earlier launch (US_ERR_CUDA) or a bounded in-kernel wait that ran out
- * (US_ERR_DEVICE_TIMEOUT). Clears the record.
+ * (US_ERR_DEVICE_TIMEOUT). Clears the record and, after a failure, the handle's split-K workspace
+ * and arrival counters (a call that gave up leaves partial sums behind).
  */
 us_status us_last_error(us_handle* h);
 
 /*
+ * Test hook for the bounded waits of the kernel (no counterpart in the paper): from now on every
+ * us_spmm on this handle leaves out the copy of the tile at `position` of the processing order
+ * (0 <= position < number of tiles) and gives up its waits after wait_us microseconds
+ * (1..2000000). Nothing is left in flight and nothing traps: the warp that waits for the missing
+ * tile times out and stops, the kernel returns, and us_last_error reports US_ERR_DEVICE_TIMEOUT.
+ * position < 0 restores normal operation.
+ */
+us_status us_debug_withhold_copy(us_handle* h, int64_t position, int64_t wait_us);
+
+/*
  * Diagnostic stage timers of the SpMM kernel (paper Sec. VII-C reports where its kernel's time
  * goes; these are the same question asked of this one). enable: 1 = record in later us_spmm
- * calls, 0 = stop, -1 = leave as is. out8 (host, may be NULL): synchronises the device, returns
- * and clears eight figures over all warps that ran since the last read -- sums of SM cycles spent
- * [0] waiting for staged tiles, [1] decoding + MMA, [2] in the reduce/store epilogue, [3] whole
- * warp lifetime; [4] the number of warps; [5] sum of cycles before a warp's first tile; [6] the
- * longest warp lifetime in cycles; [7] nanoseconds from the first warp's start to the last
- * warp's end. Recording costs a few clock reads per tile; off by default.
+ * calls, 0 = stop, -1 = leave as is. out (host, n_out >= 8 words, may be NULL): synchronises the
+ * device, returns and clears the figures of all warps that ran since the last read -- sums of SM
+ * cycles spent [0] waiting for staged tiles, [1] decoding + MMA, [2] in the reduce/store epilogue,
+ * [3] whole warp lifetime; [4] the number of warps; [5] sum of cycles before a warp's first tile;
+ * [6] the longest warp lifetime in cycles; [7] nanoseconds from the first warp's start to the last
+ * warp's end; then, as far as n_out reaches, [8..11] sums of the prologue checkpoints (cycles at
+ * which the range was known, the first copies issued, the table built, the activations staged)
+ * and from [12] five words per CTA (192 CTAs), in ns after the first warp's start: CTA start, first
+ * warp's end, activations staged, CTA end, past the wait for the stream's earlier work.
+ * Recording costs a few clock reads per tile; off by default.
  */
-us_status us_stage_timers(us_handle* h, int32_t enable, uint64_t* out8);
+us_status us_stage_timers(us_handle* h, int32_t enable, uint64_t* out, int32_t n_out);
 
 /* Frees device and host memory. NULL is accepted. */
 us_status us_destroy(us_handle* h);

@@ -23,7 +23,7 @@ US_ENCODE_SORT_ROWS = 2
 US_ENCODE_PAIR_ROWS = 4
 
 EXPORTS = ["us_encode", "us_get_stats", "us_decode", "us_get_row_order", "us_spmm", "us_spmm_static_scratch",
-           "us_last_error", "us_stage_timers", "us_destroy", "us_spmm_bytes", "us_launch_info", "us_status_string"]
+           "us_last_error", "us_debug_withhold_copy", "us_stage_timers", "us_destroy", "us_spmm_bytes", "us_launch_info", "us_status_string"]
 
 
 class us_format(ctypes.Structure):
@@ -48,7 +48,8 @@ _lib.us_spmm.argtypes = [_vp, _vp, ctypes.c_int32, _vp, _vp, _vp]
 _lib.us_last_error.argtypes = [_vp]
 _lib.us_spmm_static_scratch.argtypes = [_vp, _vp, ctypes.c_int32, _vp, _vp, _vp]
 _lib.us_destroy.argtypes = [_vp]
-_lib.us_stage_timers.argtypes = [_vp, ctypes.c_int32, _vp]
+_lib.us_stage_timers.argtypes = [_vp, ctypes.c_int32, _vp, ctypes.c_int32]
+_lib.us_debug_withhold_copy.argtypes = [_vp, ctypes.c_int64, ctypes.c_int64]
 _lib.us_spmm_bytes.argtypes = [_vp, ctypes.c_int32, ctypes.c_int32]
 _lib.us_spmm_bytes.restype = ctypes.c_int64
 _lib.us_launch_info.argtypes = [_vp, ctypes.c_int32] + [ctypes.POINTER(ctypes.c_int32)] * 3
@@ -134,15 +135,28 @@ def us_last_error(h: int) -> int:
     return int(_lib.us_last_error(h))
 
 
-def us_stage_timers(h: int, enable: int = -1, read: bool = False):
+def us_debug_withhold_copy(h: int, position: int, wait_us: int = 1000):
+    """Test hook: later us_spmm calls on the handle never copy the tile at `position` and bound
+    their waits to wait_us microseconds (position < 0: back to normal)."""
+    _check(_lib.us_debug_withhold_copy(h, int(position), int(wait_us)), "us_debug_withhold_copy")
+
+
+def us_stage_timers(h: int, enable: int = -1, read: bool = False, per_cta: int = 0):
     """Switch the kernel's stage timers on/off; with read=True return (and clear) the sums
     {wait, decode, epilogue, lifetime, prologue} in SM cycles, the number of warps, the
-    longest warp lifetime and the first-start-to-last-end span in ns."""
-    out = (ctypes.c_uint64 * 8)() if read else None
-    _check(_lib.us_stage_timers(h, int(enable), out), "us_stage_timers")
+    longest warp lifetime and the first-start-to-last-end span in ns; with per_cta = n also the
+    prologue checkpoints and, for the first n CTAs, the time stamps (start, first warp end,
+    activations staged, end, past the dependency wait) in ns."""
+    n = 8 + (4 + 5 * per_cta if per_cta else 0)
+    out = (ctypes.c_uint64 * n)() if read else None
+    _check(_lib.us_stage_timers(h, int(enable), out, n if read else 0), "us_stage_timers")
     if read:
-        return dict(zip(("wait", "decode", "epilogue", "lifetime", "warps", "prologue", "max_lifetime", "span_ns"),
-                        [int(v) for v in out]))
+        d = dict(zip(("wait", "decode", "epilogue", "lifetime", "warps", "prologue", "max_lifetime", "span_ns"),
+                     [int(v) for v in out[:8]]))
+        if per_cta:
+            d["checkpoints"] = [int(v) for v in out[8:12]]
+            d["ctas"] = [tuple(int(v) for v in out[12 + 5 * c: 17 + 5 * c]) for c in range(per_cta)]
+        return d
     return None
 
 

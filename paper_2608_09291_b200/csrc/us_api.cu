@@ -1,5 +1,6 @@
 // C ABI of the library (declared in include/unionsparse.h): handle management, upload, launch.
 #include <algorithm>
+#include <atomic>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -31,31 +32,33 @@ struct us_handle {
     uint32_t* d_err = nullptr;
     unsigned long long* d_timers = nullptr;
     bool timers_on = false;
+    size_t acc_bytes = 0, cnt_bytes = 0;
+    uint32_t withhold = 0xFFFFFFFFu;   // test hook (us_debug_withhold_copy)
+    uint32_t wait_ns_hi = 2000000u;    // bounded waits: ~2 s
     cudaError_t sticky = cudaSuccess;
 };
 
 namespace {
 
-constexpr int kMinWarps = 2;
 
 int nt_for(int N) { return N <= 8 ? 1 : N <= 16 ? 2 : N <= 32 ? 4 : 8; }
 int class_of(int nt) { return nt == 1 ? 0 : nt == 2 ? 1 : nt == 4 ? 2 : 3; }
 
-// Tuning knobs, overridable from the environment (read once per process) for experiments.
+// Experiment knobs, overridable from the environment (read once per process). Everything else the
+// plan decides from the shape.
 int env_int(const char* name, int fallback)
 {
     const char* v = std::getenv(name);
     return (v && *v) ? std::atoi(v) : fallback;
 }
-int x_budget() { static int v = env_int("US_X_BUDGET_KB", 0) * 1024; return v; }           // int8 X of one K range; 0 = automatic
-int local_acc_budget() { static int v = env_int("US_LOCAL_ACC_KB", 32) * 1024; return v; }  // local strip sums
-int stages_knob() { static int v = env_int("US_STAGES", 0); return v; }     // ring slots per warp, 0 = automatic
-int lut_rep_knob() { static int v = env_int("US_LUT_REP", 0); return v; }   // selector-table copies, 0 = automatic
 int pdl_knob() { static int v = env_int("US_PDL", 1); return v; }          // programmatic dependent launch
-int coresident_tiles_knob() { static int v = env_int("US_CORESIDENT_TILES", 16); return v; }
-int local_acc_cap() { static int v = env_int("US_LOCAL_ACC_CAP_KB", 48) * 1024; return v; }
-int coresident_knob() { static int v = env_int("US_CORESIDENT", 1); return v; }  // small problems: half an SM per CTA
+int stages_knob() { static int v = env_int("US_STAGES", 0); return v; }    // ring slots per warp, 0 = automatic
 int max_warps() { static int v = std::min(16, std::max(2, env_int("US_MAX_WARPS", 16))); return v; }
+int coresident_knob() { static int v = env_int("US_CORESIDENT", 1); return v; }  // small problems: half an SM per CTA
+constexpr int kLocalAccBudget = 32 * 1024;   // local strip sums a K-range width is chosen with
+constexpr int kLocalAccCap = 48 * 1024;      // ... and what is taken if nothing fits that
+constexpr int kMinWarps = 12;                // warps the automatic K-range choice keeps room for
+constexpr int kCoresidentTiles = 16;         // most tiles per CTA for the half-SM plan
 
 struct LaunchGeom {
     int nt, cls, warps, stages, smem, lut_rep;
@@ -68,9 +71,6 @@ struct LaunchGeom {
 // Returns the range length of the split into the fewest equal ranges, not fewer than min_ranges,
 // that still leaves room for min_warps one-slot warps (measured: 15 warps and one range beat
 // 16 warps and two ranges by 25 % on a 13824 x 5120 matrix at N = 16).
-int xp_knob() { static int v = env_int("US_PACKED_X", 1); return v; }   // 0 off, 1 automatic, 2 whenever possible
-bool plan_debug() { static int v = env_int("US_PLAN_DEBUG", 0); return v != 0; }
-int min_warps_knob() { static int v = env_int("US_MIN_WARPS", 12); return v; }
 // Shared memory of one K range's activations: int8 (one byte per token and k, 32 bytes of pad per
 // token row) or packed (half of that).
 int64_t x_bytes(int nt, int64_t G, int K_L, bool xp)
@@ -81,18 +81,14 @@ int64_t x_bytes(int nt, int64_t G, int K_L, bool xp)
 int segs_per_range(const us::HostMatrix& hm, int nt, int limit, int64_t min_ranges, bool xp)
 {
     const int64_t n_segs = hm.n_segs;
-    if (x_budget() > 0) {
-        const int g = (x_budget() / (nt * 8) - 32) / hm.fmt.K_L;
-        return (int)std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(g, n_segs), (n_segs + min_ranges - 1) / min_ranges));
-    }
     const int slot = (int)((hm.max_item_bytes + 256u + 127u) & ~127u);
-    const int acc = nt * 512 * 2 <= local_acc_budget() ? local_acc_budget() : 0;
+    const int acc = nt * 512 * 2 <= kLocalAccBudget ? kLocalAccBudget : 0;
     const int other = 256 * 8 * 4 + (int)us::kLutScratchBytes + acc + 2 * us::kOffTable * 4 + 1024;
     for (int64_t r = std::max<int64_t>(1, min_ranges); r <= n_segs; ++r) {
         // A single range is worth more (no partial sums leave the CTA when the cuts fall on strip
         // boundaries): it may cost two more warps. Measured on 4096 x 11008, N = 8: one range with
         // 15 warps 9.8 us, two ranges with 16 warps 14.7 us.
-        const int want = std::min(max_warps(), r == 1 ? std::min(10, min_warps_knob()) : min_warps_knob());
+        const int want = std::min(max_warps(), r == 1 ? std::min(10, kMinWarps) : kMinWarps);
         const int64_t G = (n_segs + r - 1) / r;
         const int64_t xb = x_bytes(nt, G, hm.fmt.K_L, xp) + G * nt * 32;
         if ((limit - other - xb) / slot >= want) return (int)G;
@@ -129,25 +125,26 @@ bool plan_launch(const us_handle* h, int N, LaunchGeom* g)
         const int w8 = std::max(warps_for(1), warps_for(2));
         // 32 copies only for long-running CTAs (measured: 1 % faster on the 70B-shaped FFN, but the
         // 4096 x 4096 case -- about one tile per warp -- loses 5 % to the bigger table)
-        const bool long_run = (h->host.n_items + 147) / 148 >= 4 * (int64_t)w8;
+        const int64_t n_cta = h->sm_count > 0 ? h->sm_count : 148;
+        const bool long_run = (h->host.n_items + n_cta - 1) / n_cta >= 4 * (int64_t)w8;
         if (w32 >= w8 && long_run) { lut_rep = 32; fixed_base = fixed_for(32); } else { lut_rep = 8; }
-        if (lut_rep_knob() == 8 || lut_rep_knob() == 32) { lut_rep = lut_rep_knob(); fixed_base = fixed_for(lut_rep); }
     }
     int stages = stages_knob() > 0 ? stages_knob() : (warps_for(1) >= warps_for(2) + 3 ? 1 : 2);
     int warps = warps_for(stages);
-    if (warps < kMinWarps) return false;
+    if (warps < 2) return false;
     // Small problems at N <= 8 (a CTA sees about a tile per warp): take at most half an SM -- shared
     // memory and registers -- with one slot per warp, so that the next launch's CTA moves in beside
     // this one and runs its latency-bound prologue (parameters, offsets, first tile copies, table)
     // under this one's work; with one CTA per SM, programmatic dependent launch alone hides only the
     // launch latency, because all CTAs of a launch end at about the same time.
     // Measured on 4096 x 4096, N = 8: 6.6 -> 5.7 us; not worth it from ~20 tiles per CTA on.
-    const int64_t per_cta = (h->host.n_items + 147) / 148;
+    const int64_t n_cta = h->sm_count > 0 ? h->sm_count : 148;
+    const int64_t per_cta = (h->host.n_items + n_cta - 1) / n_cta;
     int fixed = fixed_base + 32 * stages * 8;
     // (N = 9..16 too, where the plan stages X packed and in local mode: that kernel is as lean.)
     // (Tried at N = 32 as well: 8 warps per CTA, slower.)
     const bool co_class = g->nt == 1 || (g->nt == 2 && g->xp && s_local > 0);
-    if (coresident_knob() && co_class && per_cta <= coresident_tiles_knob() && stages_knob() == 0 && lut_rep_knob() == 0) {
+    if (coresident_knob() && co_class && per_cta <= kCoresidentTiles && stages_knob() == 0) {
         const int half = 228 * 1024 / 2 - 1024 - 512;   // per SM: 228 KB, 1 KB reserved per CTA
         const int fixed8 = fixed_for(8) + 32 * 8;
         int w = std::min(g->nt == 1 ? h->co_warps : h->co_warps2, max_warps());
@@ -185,10 +182,8 @@ void plan_classes(us_handle* h, int n_cta, std::vector<uint32_t> (&sched)[4])
                     if (G <= 1) break;
                     us::make_schedule(h->host, n_cta, G, out, &worst);
                     const int need = worst * nt * 512;
-                    if (plan_debug())
-                        fprintf(stderr, "[unionsparse] plan nt=%d%s: G=%d needs %d local strips\n", nt, xp ? " packed X" : "", G, worst);
-                    if (pass == 0 && need <= local_acc_budget()) { *s_local = worst; return G; }
-                    if (pass == 1 && need <= local_acc_cap()) {
+                    if (pass == 0 && need <= kLocalAccBudget) { *s_local = worst; return G; }
+                    if (pass == 1 && need <= kLocalAccCap) {
                         const int slot = (int)((h->host.max_item_bytes + 256u + 127u) & ~127u);
                         const int64_t fixed = 256 * 8 * 4 + (int64_t)us::kLutScratchBytes + need + 2 * us::kOffTable * 4 + 1024 +
                                               x_bytes(nt, G, h->host.fmt.K_L, xp) + (int64_t)G * nt * 32;
@@ -212,11 +207,11 @@ void plan_classes(us_handle* h, int n_cta, std::vector<uint32_t> (&sched)[4])
         // ranges become one); 5120 x 5120 12.0 -> 9.4 us (one range either way, but a CTA's share is
         // small and the staging pass and the freed shared memory count for more than the decode);
         // 13824 x 5120 15.7 -> 16.0 us (one range either way, long decode): not taken there.
-        if (nt <= 4 && xp_knob() != 0) {
+        if (nt <= 4) {
             const int64_t n_segs = h->host.n_segs;
             const int64_t ranges = h->s_local[c] > 0 ? (n_segs + h->G[c] - 1) / h->G[c] : n_segs + 1;
             const bool small_share = nt >= 2 && (int64_t)h->host.blob.size() / std::max(1, n_cta) < 128 * 1024;
-            if (ranges > 1 || small_share || xp_knob() == 2) {
+            if (ranges > 1 || small_share) {
                 std::vector<uint32_t> alt;
                 int sl2 = 0;
                 const int G2 = local_plan(true, &alt, &sl2);
@@ -224,7 +219,7 @@ void plan_classes(us_handle* h, int n_cta, std::vector<uint32_t> (&sched)[4])
                 // (N = 32, packed against plain: 11008 x 4096 21.4 -> 18.5 us, 13824 x 5120 24.9 -> 23.6 us,
                 // 5120 x 5120 17.3 -> 18.2 us with one range; three ranges instead of eleven one-segment
                 // ranges on 4096 x 11008 were slower, 19.3 -> 26.4 us: only a single range pays)
-                if (G2 > 0 && (ranges2 == 1 || xp_knob() == 2)) {
+                if (G2 > 0 && ranges2 == 1) {
                     h->G[c] = G2; h->s_local[c] = sl2; h->xp[c] = true;
                     sched[c] = alt;
                 }
@@ -237,7 +232,6 @@ void plan_classes(us_handle* h, int n_cta, std::vector<uint32_t> (&sched)[4])
     }
 }
 
-int run_knob() { static int v = env_int("US_RUN", 0); return v; }
 template <int NT, int ST>
 cudaError_t launch_st(const us::SpmmParams& p, bool xp, int grid, int block, int smem, cudaStream_t st)
 {
@@ -328,6 +322,71 @@ cudaError_t upload(T** dst, const void* src, size_t bytes)
     return bytes ? cudaMemcpy(*dst, src, bytes, cudaMemcpyHostToDevice) : cudaSuccess;
 }
 
+
+// Argument checks shared by the two SpMM entry points.
+us_status check_spmm_args(const us_handle* h, const void* X, int32_t N, const void* x_scale, const void* Y)
+{
+    if (!h || !X || !Y || N < 1 || N > h->max_N) return US_ERR_INVALID_ARG;
+    if (!h->on_device) return US_ERR_UNSUPPORTED;
+    if (x_scale && !h->d_w_scale) return US_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(X) % 16) return US_ERR_INVALID_ARG;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return US_ERR_CUDA;
+    if (dev != h->device) return US_ERR_INVALID_ARG;   // the handle's arrays live on another GPU
+    return US_OK;
+}
+
+// Fills the kernel parameters and launches: the one code path behind us_spmm and
+// us_spmm_static_scratch (they differ only in where the split-K scratch lives).
+us_status enqueue_spmm(us_handle* h, const void* X, int32_t N, const void* x_scale, void* Y, cudaStream_t st,
+                       int32_t* acc, uint32_t* cnt, bool timers)
+{
+    LaunchGeom g;
+    if (!plan_launch(h, N, &g)) return US_ERR_UNSUPPORTED;
+    const us::HostMatrix& hm = h->host;
+    us::SpmmParams p;
+    p.blob = h->d_blob; p.item_off = h->d_item_off;
+    std::memcpy(p.cta_begin, h->cta_begin[g.cls].data(), h->cta_begin[g.cls].size() * sizeof(uint32_t));
+    p.G = h->G[g.cls]; p.s_local = h->s_local[g.cls]; p.lut_rep = g.lut_rep;
+    {
+        const int64_t n_kr = (hm.n_segs + p.G - 1) / p.G;
+        const int64_t g_last = hm.n_segs - (n_kr - 1) * p.G;
+        auto magic = [](uint64_t d) { return ((1ull << 40) / d) + 1ull; };
+        p.mg_g = magic((uint64_t)p.G);
+        p.mg_glast = magic((uint64_t)g_last);
+        p.mg_krs = magic((uint64_t)hm.n_strips * (uint64_t)p.G);
+        // Claim runs of up to a whole strip's segments of the range (the partial sums of a run stay
+        // in registers; the kernel shortens the runs towards the end of a CTA's range), but never
+        // so long that a CTA's warps run out of runs to share.
+        const int64_t per_cta = std::max<int64_t>(1, hm.n_items / std::max(1, h->sm_count));
+        const int balanced = (int)std::max<int64_t>(1, per_cta / (4 * (int64_t)g.warps));
+        p.run_len = std::max(1, std::min(std::min(p.G, 2 * balanced), p.G));
+    }
+    p.row_order = h->d_row_order; p.w_scale = h->d_w_scale;
+    p.X = static_cast<const uint8_t*>(X);
+    p.x_scale = static_cast<const uint16_t*>(x_scale);
+    p.Y = Y; p.acc = acc; p.cnt = cnt; p.err = h->d_err;
+    p.timers = timers ? h->d_timers : nullptr;
+    p.M = (int32_t)hm.M; p.K = (int32_t)hm.K; p.N = N;
+    p.n_strips = (int32_t)hm.n_strips; p.n_segs = (int32_t)hm.n_segs;
+    p.mask_rows = hm.mask_rows; p.K_L = hm.fmt.K_L;
+    p.slot_bytes = g.slot_bytes;
+    p.x_fast = (hm.K % 32 == 0) ? 2 : (hm.K % 8 == 0) ? 1 : 0;
+    p.fp16_out = x_scale ? 1 : 0;
+    p.wait_ns_hi = h->wait_ns_hi;
+    p.withhold = h->withhold;
+
+    cudaError_t e;
+    switch (g.nt) {
+        case 1: e = launch_nt<1>(p, g.xp, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
+        case 2: e = launch_nt<2>(p, g.xp, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
+        case 4: e = launch_nt<4>(p, g.xp, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
+        default: e = launch_nt<8>(p, g.xp, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
+    }
+    if (e != cudaSuccess) { h->sticky = e; return US_ERR_CUDA; }
+    return US_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -338,10 +397,20 @@ us_status us_encode(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_sca
     if (out) *out = nullptr;
     if (!W || !out || M <= 0 || K <= 0 || max_N < 1 || max_N > 64) return US_ERR_INVALID_ARG;
     if (M > 0x7FFFFFF0ll || K > 0x7FFFFFF0ll) return US_ERR_INVALID_ARG;
-    us_format f = fmt ? *fmt : us_format{16, us::default_K_L(M, K), 2, 1};
     us_handle* h = new (std::nothrow) us_handle();
     if (!h) return US_ERR_ALLOC;
     h->max_N = max_N;
+    const bool host_only = (flags & US_ENCODE_HOST_ONLY) != 0;
+    cudaError_t e = cudaSuccess;
+    if (!host_only) {
+        e = cudaGetDevice(&h->device);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device);
+        if (e != cudaSuccess) { delete h; return US_ERR_CUDA; }
+        if (h->sm_count > us::kMaxCtas) h->sm_count = us::kMaxCtas;
+    }
+    const int n_cta = h->sm_count > 0 ? h->sm_count : 148;   // host-only handles plan for a 148-SM part
+    us_format f = fmt ? *fmt : us_format{16, us::default_K_L(M, K, n_cta), 2, 1};
     us_status s;
     try {
         s = us::encode_host(W, M, K, w_scale, f, flags, 0, &h->host);
@@ -349,29 +418,32 @@ us_status us_encode(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_sca
         s = US_ERR_ALLOC;
     }
     if (s != US_OK) { delete h; return s; }
-    if (h->host.n_items >= (1 << 24) || h->host.n_strips * h->host.n_segs >= (1 << 24) || h->host.n_segs >= (1 << 16)) {
-        delete h;
-        return US_ERR_UNSUPPORTED;  // the kernel's index arithmetic assumes fewer tiles
+    const us::HostMatrix& hm = h->host;
+    if (!hm.kernel_layout) {   // a format without a kernel: statistics and decoding only
+        *out = h;
+        return US_OK;
     }
-    if (flags & US_ENCODE_HOST_ONLY) {
-        std::vector<uint32_t> sched[4];
-        plan_classes(h, 148, sched);
+    // the kernel's index arithmetic (exact division by multiplication) needs u * d < 2^40 for every
+    // position u < n_items and divisor d <= n_items
+    if (hm.n_items >= (1 << 20) || hm.n_segs >= (1 << 16)) {
+        delete h;
+        return US_ERR_UNSUPPORTED;
+    }
+    std::vector<uint32_t> sched[4];
+    plan_classes(h, n_cta, sched);
+    if (host_only) {
         *out = h;
         return US_OK;
     }
 
-    cudaError_t e = cudaGetDevice(&h->device);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device);
-    if (e == cudaSuccess && h->sm_count > us::kMaxCtas) h->sm_count = us::kMaxCtas;
-    if (e == cudaSuccess) e = enable_large_smem(h->max_smem);
+    e = enable_large_smem(h->max_smem);
     if (e == cudaSuccess) {
         // Two N <= 8 CTAs share the SM's 64 K registers (allocated 8 per thread at a time).
         int regs = 0;
         // (the stage-timer builds need more and simply do not share an SM)
-        for (const void* f : {(const void*)us::us_spmm_kernel<1, 1, true, false>, (const void*)us::us_spmm_kernel<1, 1, false, false>}) {
+        for (const void* fn : {(const void*)us::us_spmm_kernel<1, 1, true, false>, (const void*)us::us_spmm_kernel<1, 1, false, false>}) {
             cudaFuncAttributes fa;
-            e = cudaFuncGetAttributes(&fa, f);
+            e = cudaFuncGetAttributes(&fa, fn);
             if (e != cudaSuccess) break;
             regs = std::max(regs, fa.numRegs);
         }
@@ -379,25 +451,21 @@ us_status us_encode(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_sca
         cudaFuncAttributes fa2;
         if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa2, (const void*)us::us_spmm_kernel<2, 1, true, false, true>);
         if (e == cudaSuccess) h->co_warps2 = 32768 / (32 * ((fa2.numRegs + 7) / 8 * 8));
-
     }
     if (e != cudaSuccess) { delete h; return US_ERR_CUDA; }
 
-    const us::HostMatrix& hm = h->host;
-    std::vector<uint32_t> sched[4];
-    plan_classes(h, h->sm_count, sched);
     const int nt_max = nt_for(max_N);
-    const size_t acc_bytes = (size_t)hm.n_strips * nt_max * 128 * sizeof(int32_t);
-    const size_t cnt_bytes = (size_t)hm.n_strips * sizeof(uint32_t);
+    h->acc_bytes = (size_t)hm.n_strips * nt_max * 128 * sizeof(int32_t);
+    h->cnt_bytes = (size_t)hm.n_strips * sizeof(uint32_t);
     e = upload(&h->d_blob, hm.blob.data(), hm.blob.size());
     if (e == cudaSuccess) e = upload(&h->d_item_off, hm.item_off.data(), hm.item_off.size() * 4);
     for (int c = 0; c < 4; ++c) h->cta_begin[c] = sched[c];
     if (e == cudaSuccess) e = upload(&h->d_row_order, hm.row_order.data(), hm.row_order.size() * 4);
     if (e == cudaSuccess && !hm.w_scale.empty()) e = upload(&h->d_w_scale, hm.w_scale.data(), hm.w_scale.size() * 2);
-    if (e == cudaSuccess) e = cudaMalloc((void**)&h->d_acc, acc_bytes);
-    if (e == cudaSuccess) e = cudaMemset(h->d_acc, 0, acc_bytes);
-    if (e == cudaSuccess) e = cudaMalloc((void**)&h->d_cnt, cnt_bytes);
-    if (e == cudaSuccess) e = cudaMemset(h->d_cnt, 0, cnt_bytes);
+    if (e == cudaSuccess) e = cudaMalloc((void**)&h->d_acc, h->acc_bytes);
+    if (e == cudaSuccess) e = cudaMemset(h->d_acc, 0, h->acc_bytes);
+    if (e == cudaSuccess) e = cudaMalloc((void**)&h->d_cnt, h->cnt_bytes);
+    if (e == cudaSuccess) e = cudaMemset(h->d_cnt, 0, h->cnt_bytes);
     if (e == cudaSuccess) e = cudaMalloc((void**)&h->d_err, 16);
     if (e == cudaSuccess) e = cudaMemset(h->d_err, 0, 16);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
@@ -435,6 +503,10 @@ us_status us_decode(const us_handle* h, int8_t* W_out)
 us_status us_get_row_order(const us_handle* h, int32_t* perm_out)
 {
     if (!h || !perm_out) return US_ERR_INVALID_ARG;
+    if (!h->host.kernel_layout) {   // the paper's layout keeps the rows where they are
+        for (int64_t r = 0; r < h->host.Mp; ++r) perm_out[r] = r < h->host.M ? (int32_t)r : -1;
+        return US_OK;
+    }
     std::memcpy(perm_out, h->host.row_order.data(), h->host.row_order.size() * sizeof(int32_t));
     return US_OK;
 }
@@ -443,6 +515,7 @@ us_status us_launch_info(const us_handle* h, int32_t N, int32_t* grid, int32_t* 
                          int32_t* smem_bytes)
 {
     if (!h || N < 1 || N > h->max_N) return US_ERR_INVALID_ARG;
+    if (!h->host.kernel_layout) return US_ERR_UNSUPPORTED;
     LaunchGeom g;
     if (!plan_launch(h, N, &g)) return US_ERR_UNSUPPORTED;
     if (grid) *grid = h->sm_count > 0 ? h->sm_count : 148;
@@ -453,55 +526,9 @@ us_status us_launch_info(const us_handle* h, int32_t N, int32_t* grid, int32_t* 
 
 us_status us_spmm(us_handle* h, const void* X, int32_t N, const void* x_scale, void* Y, void* stream)
 {
-    if (!h || !X || !Y || N < 1 || N > h->max_N) return US_ERR_INVALID_ARG;
-    if (!h->on_device) return US_ERR_UNSUPPORTED;
-    if (x_scale && !h->d_w_scale) return US_ERR_INVALID_ARG;
-    if (reinterpret_cast<uintptr_t>(X) % 16) return US_ERR_INVALID_ARG;
-    LaunchGeom g;
-    if (!plan_launch(h, N, &g)) return US_ERR_UNSUPPORTED;
-
-    const us::HostMatrix& hm = h->host;
-    us::SpmmParams p;
-    p.blob = h->d_blob; p.item_off = h->d_item_off;
-    std::memcpy(p.cta_begin, h->cta_begin[g.cls].data(), h->cta_begin[g.cls].size() * sizeof(uint32_t));
-    p.G = h->G[g.cls]; p.s_local = h->s_local[g.cls]; p.lut_rep = g.lut_rep;
-    {
-        const int64_t n_kr = (hm.n_segs + p.G - 1) / p.G;
-        const int64_t g_last = hm.n_segs - (n_kr - 1) * p.G;
-        auto magic = [](uint64_t d) { return ((1ull << 40) / d) + 1ull; };
-        p.mg_g = magic((uint64_t)p.G);
-        p.mg_glast = magic((uint64_t)g_last);
-        p.mg_krs = magic((uint64_t)hm.n_strips * (uint64_t)p.G);
-        // Claim runs of up to a whole strip's segments of the range (the partial sums of a run stay
-        // in registers; the kernel shortens the runs towards the end of a CTA's range), but never
-        // so long that a CTA's warps run out of runs to share.
-        const int64_t per_cta = std::max<int64_t>(1, hm.n_items / std::max(1, h->sm_count));
-        const int balanced = (int)std::max<int64_t>(1, per_cta / (4 * (int64_t)g.warps));
-        const int want = run_knob() > 0 ? run_knob() : std::min(p.G, 2 * balanced);
-        p.run_len = std::max(1, std::min(want, p.G));
-    }
-    p.row_order = h->d_row_order; p.w_scale = h->d_w_scale;
-    p.X = static_cast<const uint8_t*>(X);
-    p.x_scale = static_cast<const uint16_t*>(x_scale);
-    p.Y = Y; p.acc = h->d_acc; p.cnt = h->d_cnt; p.err = h->d_err;
-    p.timers = h->timers_on ? h->d_timers : nullptr;
-    p.M = (int32_t)hm.M; p.K = (int32_t)hm.K; p.N = N;
-    p.n_strips = (int32_t)hm.n_strips; p.n_segs = (int32_t)hm.n_segs;
-    p.nkb = hm.nkb; p.mask_rows = hm.mask_rows; p.K_L = hm.fmt.K_L;
-    p.slot_bytes = g.slot_bytes;
-    p.x_fast = (hm.K % 32 == 0) ? 2 : (hm.K % 8 == 0) ? 1 : 0;
-    p.fp16_out = x_scale ? 1 : 0;
-
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    cudaError_t e;
-    switch (g.nt) {
-        case 1: e = launch_nt<1>(p, g.xp, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
-        case 2: e = launch_nt<2>(p, g.xp, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
-        case 4: e = launch_nt<4>(p, g.xp, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
-        default: e = launch_nt<8>(p, g.xp, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
-    }
-    if (e != cudaSuccess) { h->sticky = e; return US_ERR_CUDA; }
-    return US_OK;
+    const us_status s = check_spmm_args(h, X, N, x_scale, Y);
+    if (s != US_OK) return s;
+    return enqueue_spmm(h, X, N, x_scale, Y, static_cast<cudaStream_t>(stream), h->d_acc, h->d_cnt, h->timers_on);
 }
 
 // ---- us_spmm_static_scratch: the SpMM with its scratch in a fixed device array ------------------
@@ -512,78 +539,36 @@ static __device__ __align__(256) unsigned char g_static_scratch[US_STATIC_SCRATC
 
 namespace {
 constexpr int kMaxDevices = 64;
-void* g_scratch_addr[kMaxDevices] = {nullptr};
+std::atomic<void*> g_scratch_addr[kMaxDevices];   // zero-initialised; one look-up per device
 }  // namespace
 
 us_status us_spmm_static_scratch(us_handle* h, const void* X, int32_t N, const void* x_scale, void* Y,
                                  void* stream)
 {
-    if (!h || !X || !Y || N < 1 || N > h->max_N) return US_ERR_INVALID_ARG;
-    if (!h->on_device) return US_ERR_UNSUPPORTED;
-    if (x_scale && !h->d_w_scale) return US_ERR_INVALID_ARG;
-    if (reinterpret_cast<uintptr_t>(X) % 16) return US_ERR_INVALID_ARG;
-    LaunchGeom g;
-    if (!plan_launch(h, N, &g)) return US_ERR_UNSUPPORTED;
-
+    const us_status s = check_spmm_args(h, X, N, x_scale, Y);
+    if (s != US_OK) return s;
     const us::HostMatrix& hm = h->host;
     // scratch the kernel needs: INT32 strip sums, then one arrival counter per strip
-    const size_t acc_bytes = (size_t)hm.n_strips * g.nt * 128 * sizeof(int32_t);
+    const size_t acc_bytes = (size_t)hm.n_strips * nt_for(N) * 128 * sizeof(int32_t);
     const size_t cnt_bytes = (size_t)hm.n_strips * sizeof(uint32_t);
     if (acc_bytes + cnt_bytes > (size_t)US_STATIC_SCRATCH_BYTES) return US_ERR_SCRATCH_TOO_SMALL;
 
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess) return US_ERR_CUDA;
-    if (dev != h->device || dev < 0 || dev >= kMaxDevices) return US_ERR_INVALID_ARG;
-    if (!g_scratch_addr[dev]) {  // set-up, once per device, with that device current
-        void* ptr = nullptr;
+    const int dev = h->device;   // checked above: it is the current device
+    if (dev < 0 || dev >= kMaxDevices) return US_ERR_INVALID_ARG;
+    void* ptr = g_scratch_addr[dev].load(std::memory_order_acquire);
+    if (!ptr) {  // set-up, once per device, with that device current (threads racing here all
+                 // look up the same address)
         const cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
         if (e != cudaSuccess || !ptr) { h->sticky = e; return US_ERR_CUDA; }
-        g_scratch_addr[dev] = ptr;
+        g_scratch_addr[dev].store(ptr, std::memory_order_release);
     }
-    unsigned char* scratch = static_cast<unsigned char*>(g_scratch_addr[dev]);
+    unsigned char* scratch = static_cast<unsigned char*>(ptr);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // The array keeps the previous call's contents: sums and counters must start at zero.
-    cudaError_t e = cudaMemsetAsync(scratch, 0, acc_bytes + cnt_bytes, st);
+    const cudaError_t e = cudaMemsetAsync(scratch, 0, acc_bytes + cnt_bytes, st);
     if (e != cudaSuccess) { h->sticky = e; return US_ERR_CUDA; }
-
-    us::SpmmParams p;
-    p.blob = h->d_blob; p.item_off = h->d_item_off;
-    std::memcpy(p.cta_begin, h->cta_begin[g.cls].data(), h->cta_begin[g.cls].size() * sizeof(uint32_t));
-    p.G = h->G[g.cls]; p.s_local = h->s_local[g.cls]; p.lut_rep = g.lut_rep;
-    {
-        const int64_t n_kr = (hm.n_segs + p.G - 1) / p.G;
-        const int64_t g_last = hm.n_segs - (n_kr - 1) * p.G;
-        auto magic = [](uint64_t d) { return ((1ull << 40) / d) + 1ull; };
-        p.mg_g = magic((uint64_t)p.G);
-        p.mg_glast = magic((uint64_t)g_last);
-        p.mg_krs = magic((uint64_t)hm.n_strips * (uint64_t)p.G);
-        const int64_t per_cta = std::max<int64_t>(1, hm.n_items / std::max(1, h->sm_count));
-        const int balanced = (int)std::max<int64_t>(1, per_cta / (4 * (int64_t)g.warps));
-        const int want = run_knob() > 0 ? run_knob() : std::min(p.G, 2 * balanced);
-        p.run_len = std::max(1, std::min(want, p.G));
-    }
-    p.row_order = h->d_row_order; p.w_scale = h->d_w_scale;
-    p.X = static_cast<const uint8_t*>(X);
-    p.x_scale = static_cast<const uint16_t*>(x_scale);
-    p.Y = Y;
-    p.acc = reinterpret_cast<int32_t*>(scratch);
-    p.cnt = reinterpret_cast<uint32_t*>(scratch + acc_bytes);
-    p.err = h->d_err;
-    p.timers = nullptr;
-    p.M = (int32_t)hm.M; p.K = (int32_t)hm.K; p.N = N;
-    p.n_strips = (int32_t)hm.n_strips; p.n_segs = (int32_t)hm.n_segs;
-    p.nkb = hm.nkb; p.mask_rows = hm.mask_rows; p.K_L = hm.fmt.K_L;
-    p.slot_bytes = g.slot_bytes;
-    p.x_fast = (hm.K % 32 == 0) ? 2 : (hm.K % 8 == 0) ? 1 : 0;
-    p.fp16_out = x_scale ? 1 : 0;
-    switch (g.nt) {
-        case 1: e = launch_nt<1>(p, g.xp, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
-        case 2: e = launch_nt<2>(p, g.xp, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
-        case 4: e = launch_nt<4>(p, g.xp, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
-        default: e = launch_nt<8>(p, g.xp, g.stages, h->sm_count, g.warps * 32, g.smem, st); break;
-    }
-    if (e != cudaSuccess) { h->sticky = e; return US_ERR_CUDA; }
-    return US_OK;
+    return enqueue_spmm(h, X, N, x_scale, Y, st, reinterpret_cast<int32_t*>(scratch),
+                        reinterpret_cast<uint32_t*>(scratch + acc_bytes), false);
 }
 
 us_status us_last_error(us_handle* h)
@@ -593,49 +578,82 @@ us_status us_last_error(us_handle* h)
     cudaError_t e = cudaDeviceSynchronize();
     uint32_t flag = 0;
     if (e == cudaSuccess) e = cudaMemcpy(&flag, h->d_err, 4, cudaMemcpyDeviceToHost);
-    if (e == cudaSuccess && flag) cudaMemset(h->d_err, 0, 4);
+    const bool failed = flag != 0 || h->sticky != cudaSuccess || e != cudaSuccess;
+    if (failed) {
+        // A call that gave up leaves partial sums and arrival counts behind: clear them, so that the
+        // next call on this handle starts from the zeroed workspace it relies on.
+        cudaMemset(h->d_err, 0, 4);
+        cudaMemset(h->d_acc, 0, h->acc_bytes);
+        cudaMemset(h->d_cnt, 0, h->cnt_bytes);
+        cudaDeviceSynchronize();
+    }
     if (h->sticky != cudaSuccess) { e = h->sticky; h->sticky = cudaSuccess; }
-    if (e != cudaSuccess) return US_ERR_CUDA;
+    if (e != cudaSuccess) { cudaGetLastError(); return US_ERR_CUDA; }
     if (flag == us::kErrTimeout) return US_ERR_DEVICE_TIMEOUT;
     return flag ? US_ERR_CUDA : US_OK;
 }
 
-static cudaError_t reset_timers(unsigned long long* d)
-{
-    static unsigned long long z[16 + 4 * us::kMaxCtas];
-    std::memset(z, 0, sizeof(z));
-    z[7] = ~0ull;  // running minimum of the start time stamps
-    return cudaMemcpy(d, z, sizeof(z), cudaMemcpyHostToDevice);
-}
-
-us_status us_stage_timers(us_handle* h, int32_t enable, uint64_t* out8)
+us_status us_debug_withhold_copy(us_handle* h, int64_t position, int64_t wait_us)
 {
     if (!h) return US_ERR_INVALID_ARG;
     if (!h->on_device) return US_ERR_UNSUPPORTED;
-    if (!h->d_timers) {
-        if (cudaMalloc((void**)&h->d_timers, (16 + 4 * us::kMaxCtas) * sizeof(unsigned long long)) != cudaSuccess) return US_ERR_ALLOC;
-        reset_timers(h->d_timers);
+    if (position < 0) {
+        h->withhold = 0xFFFFFFFFu;
+        h->wait_ns_hi = 2000000u;
+        return US_OK;
     }
-    if (out8) {
+    if (position >= h->host.n_items || wait_us < 1 || wait_us > 2000000) return US_ERR_INVALID_ARG;
+    h->withhold = (uint32_t)position;
+    h->wait_ns_hi = (uint32_t)std::max<int64_t>(1, wait_us * 1000 / 1024);
+    return US_OK;
+}
+
+us_status us_stage_timers(us_handle* h, int32_t enable, uint64_t* out, int32_t n_out)
+{
+    if (!h || (out && n_out < 8)) return US_ERR_INVALID_ARG;
+    if (!h->on_device) return US_ERR_UNSUPPORTED;
+    const size_t bytes = us::kTimerWords * sizeof(unsigned long long);
+    if (!h->d_timers) {
+        if (cudaMalloc((void**)&h->d_timers, bytes) != cudaSuccess) return US_ERR_ALLOC;
+        cudaMemset(h->d_timers, 0, bytes);
+    }
+    if (out) {
         if (cudaDeviceSynchronize() != cudaSuccess) return US_ERR_CUDA;
-        static uint64_t t[16 + 4 * us::kMaxCtas];
-        if (cudaMemcpy(t, h->d_timers, sizeof(t), cudaMemcpyDeviceToHost) != cudaSuccess) return US_ERR_CUDA;
-        if (const char* path = std::getenv("US_TIMER_DUMP")) {
-            if (FILE* f = std::fopen(path, "a")) {
-                for (int c = 0; c < us::kMaxCtas; ++c)
-                    if (t[16 + 4 * c])
-                        std::fprintf(f, "%d %llu %llu %llu %lld\n", c, (unsigned long long)t[16 + 4 * c], (unsigned long long)t[17 + 4 * c],
-                                     (unsigned long long)t[18 + 4 * c], (long long)(t[19 + 4 * c] - t[7]));
-                std::fprintf(f, "#\n");
-                std::fclose(f);
+        std::vector<uint64_t> t((size_t)us::kTimerWords);
+        if (cudaMemcpy(t.data(), h->d_timers, bytes, cudaMemcpyDeviceToHost) != cudaSuccess) return US_ERR_CUDA;
+        // reduce the per-warp records
+        uint64_t sum[6] = {0, 0, 0, 0, 0, 0}, ck[4] = {0, 0, 0, 0}, max_life = 0, t_min = ~0ull, t_max = 0;
+        std::vector<uint64_t> cta((size_t)5 * us::kMaxCtas, 0);   // per CTA: start, first warp end, X staged, end, past the dependency wait
+        for (int c = 0; c < us::kMaxCtas; ++c) {
+            uint64_t st = ~0ull, first_end = ~0ull, xs = 0, en = 0, pw = 0;
+            for (int w = 0; w < us::kMaxWarpsPerCta; ++w) {
+                const uint64_t* R = t.data() + (size_t)us::kWarpRec * ((size_t)c * us::kMaxWarpsPerCta + w);
+                if (!R[0]) continue;
+                for (int i = 0; i < 4; ++i) sum[i] += R[1 + i];
+                sum[4] += 1;
+                sum[5] += R[5];
+                max_life = std::max(max_life, R[4]);
+                for (int i = 0; i < 4; ++i) ck[i] += R[9 + i];
+                st = std::min(st, R[6]); first_end = std::min(first_end, R[8]); xs = std::max(xs, R[7]);
+                en = std::max(en, R[8]); pw = std::max(pw, R[13]);
+            }
+            if (en) {
+                t_min = std::min(t_min, st); t_max = std::max(t_max, en);
+                cta[5 * c] = st; cta[5 * c + 1] = first_end; cta[5 * c + 2] = xs; cta[5 * c + 3] = en; cta[5 * c + 4] = pw;
             }
         }
-        for (int i = 0; i < 7; ++i) out8[i] = t[i];
-        out8[7] = t[8] > t[7] ? t[8] - t[7] : 0;   // first warp start to last warp end, ns
-        if (std::getenv("US_TIMER_DEBUG") && t[4])
-            std::fprintf(stderr, "[us] prologue checkpoints (cycles/warp): range known %.0f, copies issued %.0f, table done %.0f, X staged %.0f\n",
-                         (double)t[9] / t[4], (double)t[10] / t[4], (double)t[11] / t[4], (double)t[12] / t[4]);
-        reset_timers(h->d_timers);
+        for (int i = 0; i < 6; ++i) out[i] = sum[i];
+        out[6] = max_life;
+        out[7] = t_max > t_min ? t_max - t_min : 0;   // first warp start to last warp end, ns
+        // optional tail: prologue checkpoints, then five time stamps per CTA
+        for (int i = 8; i < n_out; ++i) {
+            const int j = i - 8;
+            uint64_t v = 0;
+            if (j < 4) v = ck[j];
+            else if (j - 4 < 5 * us::kMaxCtas) v = cta[j - 4] ? cta[j - 4] - t_min : 0;
+            out[i] = v;
+        }
+        cudaMemset(h->d_timers, 0, bytes);
     }
     if (enable >= 0) h->timers_on = enable != 0;
     return US_OK;

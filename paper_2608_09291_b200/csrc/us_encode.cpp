@@ -1,5 +1,6 @@
-// Host encoder / decoder of the lane-stream IE-BME layout (see us_host.h), statistics
-// (paper Sec. V-A storage arrays, Eq. 1) and the CTA schedule. Pure C++: no CUDA here.
+// Host encoder / decoder of the lane-stream IE-BME layout (see us_host.h), the paper's own array
+// layout for every other format, statistics (paper Sec. V-A storage arrays, Eq. 1) and the CTA
+// schedule. Pure C++: no CUDA here.
 #include <algorithm>
 #include <climits>
 #include <atomic>
@@ -104,16 +105,123 @@ void pair_rows(const int8_t* W, int64_t M, int64_t K, int threads, HostMatrix* h
 
 }  // namespace
 
-int32_t default_K_L(int64_t M, int64_t K)
+int32_t default_K_L(int64_t M, int64_t K, int n_sm)
 {
     // Large tiles keep the per-tile padding of the lane streams small; small matrices get
-    // smaller tiles so that every warp of a 148-SM part still finds work.
+    // smaller tiles so that every warp of every SM still finds work.
     // (Measured on a 4096 x 4096 matrix at 50 % sparsity: 512 beats both 256 and 1024.)
     const int64_t strips = (M + 15) / 16;
-    if (strips * ((K + 1023) / 1024) >= 148 * 16) return 1024;
-    if (strips * ((K + 511) / 512) >= 148 * 4) return 512;
+    if (n_sm <= 0) n_sm = 148;
+    if (strips * ((K + 1023) / 1024) >= (int64_t)n_sm * 16) return 1024;
+    if (strips * ((K + 511) / 512) >= (int64_t)n_sm * 4) return 512;
     return 256;
 }
+
+namespace {
+
+// ---- the paper's own array layout, any (H_L, K_L, R_A, C_A) (Sec. V-A) ---------------------------
+// Local tiles in row-block-major order; area q = a * C_A + c is the block of rows
+// [a * H_L/R_A, ...) and columns [c * K_L/C_A, ...) of the tile; one union-mask bit per position
+// of an area, row-major, leftmost column in the least significant bit of 64-bit words; for every
+// active bit the Q values of the areas go to Q consecutive streams of P_t values each.
+us_status encode_generic(const int8_t* W, int64_t M, int64_t K, const us_format& f, int threads, HostMatrix* hp)
+{
+    HostMatrix& h = *hp;
+    const int Q = f.R_A * f.C_A, hb = f.H_L / f.R_A, kb = f.K_L / f.C_A;
+    h.Mp = (M + f.H_L - 1) / f.H_L * f.H_L;
+    h.Kp = (K + f.K_L - 1) / f.K_L * f.K_L;
+    const int64_t tk = h.Kp / f.K_L, n_lt = (h.Mp / f.H_L) * tk;
+    GenericArrays& g = h.gen;
+    g.n_lt = n_lt;
+    g.words_per_lt = (int64_t)hb * kb / 64;
+    g.bitmaps.assign((size_t)(n_lt * g.words_per_lt), 0);
+    g.offsets.assign((size_t)n_lt + 1, 0);
+    std::vector<uint32_t> P((size_t)n_lt, 0);
+    std::atomic<int> bad{0};
+    std::atomic<int64_t> nnz{0};
+    auto at = [&](int64_t r, int64_t c) -> int { return (r < M && c < K) ? W[r * K + c] : 0; };
+    // pass 1: union masks and their populations
+    parallel_for(n_lt, threads, [&](int64_t t, int) {
+        const int64_t r0 = t / tk * f.H_L, c0 = t % tk * f.K_L;
+        uint64_t* bm = g.bitmaps.data() + t * g.words_per_lt;
+        uint32_t pop = 0;
+        int64_t nz = 0;
+        for (int i = 0; i < hb; ++i)
+            for (int j = 0; j < kb; ++j) {
+                bool any = false;
+                for (int q = 0; q < Q; ++q) {
+                    const int v = at(r0 + (q / f.C_A) * hb + i, c0 + (q % f.C_A) * kb + j);
+                    if (v < -8 || v > 7) bad.store(1);
+                    if (v) { any = true; ++nz; }
+                }
+                if (any) {
+                    const int64_t bit = (int64_t)i * kb + j;
+                    bm[bit >> 6] |= 1ull << (bit & 63);
+                    ++pop;
+                }
+            }
+        P[t] = pop;
+        nnz += nz;
+    });
+    if (bad.load()) return US_ERR_VALUE_RANGE;
+    uint64_t o = 0;
+    for (int64_t t = 0; t < n_lt; ++t) {
+        g.offsets[t] = (uint32_t)o;
+        o += (uint64_t)Q * P[t];
+        if (o > 0xFFFFFFFFull) return US_ERR_ALLOC;
+    }
+    g.offsets[n_lt] = (uint32_t)o;
+    g.values.assign((size_t)((o + 1) / 2), 0);
+    // pass 2: the value streams (two tiles never share a byte only when their offsets are even;
+    // an odd total would make neighbours share one, so this pass runs tile after tile)
+    for (int64_t t = 0; t < n_lt; ++t) {
+        const int64_t r0 = t / tk * f.H_L, c0 = t % tk * f.K_L;
+        const uint64_t* bm = g.bitmaps.data() + t * g.words_per_lt;
+        uint64_t rank = 0;
+        for (int64_t bit = 0; bit < (int64_t)hb * kb; ++bit) {
+            if (!((bm[bit >> 6] >> (bit & 63)) & 1)) continue;
+            const int i = (int)(bit / kb), j = (int)(bit % kb);
+            for (int q = 0; q < Q; ++q) {
+                const uint64_t idx = g.offsets[t] + (uint64_t)q * P[t] + rank;
+                const uint8_t nib = (uint8_t)at(r0 + (q / f.C_A) * hb + i, c0 + (q % f.C_A) * kb + j) & 0xF;
+                g.values[idx >> 1] |= (uint8_t)(nib << (4 * (idx & 1)));
+            }
+            ++rank;
+        }
+        h.sum_P += P[t];
+    }
+    h.nnz = nnz.load();
+    h.n_strips = h.Mp / f.H_L;
+    h.n_segs = tk;
+    return US_OK;
+}
+
+void decode_generic(const HostMatrix& h, int8_t* W_out)
+{
+    const us_format& f = h.fmt;
+    const GenericArrays& g = h.gen;
+    const int Q = f.R_A * f.C_A, hb = f.H_L / f.R_A, kb = f.K_L / f.C_A;
+    const int64_t tk = h.Kp / f.K_L;
+    for (int64_t t = 0; t < g.n_lt; ++t) {
+        const int64_t r0 = t / tk * f.H_L, c0 = t % tk * f.K_L;
+        const uint64_t* bm = g.bitmaps.data() + t * g.words_per_lt;
+        const uint64_t P = (g.offsets[t + 1] - g.offsets[t]) / (uint64_t)Q;
+        uint64_t rank = 0;
+        for (int64_t bit = 0; bit < (int64_t)hb * kb; ++bit) {
+            if (!((bm[bit >> 6] >> (bit & 63)) & 1)) continue;
+            const int i = (int)(bit / kb), j = (int)(bit % kb);
+            for (int q = 0; q < Q; ++q) {
+                const uint64_t idx = g.offsets[t] + (uint64_t)q * P + rank;
+                const int nib = (g.values[idx >> 1] >> (4 * (idx & 1))) & 0xF;
+                const int64_t r = r0 + (q / f.C_A) * hb + i, c = c0 + (q % f.C_A) * kb + j;
+                if (r < h.M && c < h.K) W_out[r * h.K + c] = (int8_t)(nib >= 8 ? nib - 16 : nib);
+            }
+            ++rank;
+        }
+    }
+}
+
+}  // namespace
 
 us_status encode_host(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_scale,
                       const us_format& fmt, uint32_t flags, int threads, HostMatrix* out)
@@ -122,12 +230,21 @@ us_status encode_host(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_s
     if (fmt.H_L <= 0 || fmt.K_L <= 0 || fmt.R_A <= 0 || fmt.C_A <= 0) return US_ERR_SHAPE;
     if (fmt.H_L % fmt.R_A || fmt.K_L % fmt.C_A) return US_ERR_SHAPE;
     if (((int64_t)(fmt.H_L / fmt.R_A) * (fmt.K_L / fmt.C_A)) % 64) return US_ERR_SHAPE;
-    if (fmt.H_L != 16 || fmt.R_A != 2 || fmt.C_A != 1 || fmt.K_L % 128 || fmt.K_L > 8192)
-        return US_ERR_UNSUPPORTED;
 
     HostMatrix& h = *out;
     h = HostMatrix();
     h.M = M; h.K = K; h.fmt = fmt;
+    h.kernel_layout = fmt.H_L == 16 && fmt.R_A == 2 && fmt.C_A == 1 && fmt.K_L % 128 == 0 && fmt.K_L <= 8192;
+    if (!h.kernel_layout) {
+        // a valid IE-BME format without a kernel: the paper's arrays, for statistics and decoding
+        if (!(flags & US_ENCODE_HOST_ONLY)) return US_ERR_UNSUPPORTED;
+        if (flags & (US_ENCODE_SORT_ROWS | US_ENCODE_PAIR_ROWS)) return US_ERR_UNSUPPORTED;
+        if ((int64_t)fmt.H_L * fmt.K_L > (1 << 24)) return US_ERR_UNSUPPORTED;
+        if (w_scale) h.w_scale.assign(w_scale, w_scale + M);
+        us_status st = encode_generic(W, M, K, fmt, threads, &h);
+        if (st != US_OK) h = HostMatrix();
+        return st;
+    }
     h.Mp = (M + 15) / 16 * 16;
     h.Kp = (K + fmt.K_L - 1) / fmt.K_L * fmt.K_L;
     h.nkb = fmt.K_L / 32;
@@ -241,6 +358,7 @@ us_status encode_host(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_s
 void decode_host(const HostMatrix& h, int8_t* W_out)
 {
     std::memset(W_out, 0, (size_t)(h.M * h.K));
+    if (!h.kernel_layout) { decode_generic(h, W_out); return; }
     const int nkb = h.nkb, mask_rows = h.mask_rows, K_L = h.fmt.K_L;
     for (int64_t t = 0; t < h.n_items; ++t) {
         const int64_t rb = t / h.n_segs, sg = t % h.n_segs;
@@ -273,12 +391,19 @@ void fill_stats(const HostMatrix& h, us_stats* st)
     const int Q = h.fmt.R_A * h.fmt.C_A;
     st->M = h.M; st->K = h.K; st->Mp = h.Mp; st->Kp = h.Kp;
     st->nnz = h.nnz;
-    st->n_tiles = h.n_items;
     st->sum_P = h.sum_P;
     st->bytes_payload = ((int64_t)Q * h.sum_P + 1) / 2;
-    st->bytes_payload_padded = h.bytes_payload_padded;
-    st->bytes_bitmap = h.n_items * (int64_t)h.mask_rows * 128;
-    st->bytes_offsets = 4 * (h.n_items + 1);
+    if (h.kernel_layout) {
+        st->n_tiles = h.n_items;
+        st->bytes_payload_padded = h.bytes_payload_padded;
+        st->bytes_bitmap = h.n_items * (int64_t)h.mask_rows * 128;
+        st->bytes_offsets = 4 * (h.n_items + 1);
+    } else {
+        st->n_tiles = h.gen.n_lt;
+        st->bytes_payload_padded = (int64_t)h.gen.values.size();
+        st->bytes_bitmap = 8 * h.gen.n_lt * h.gen.words_per_lt;
+        st->bytes_offsets = 4 * (h.gen.n_lt + 1);
+    }
     st->bytes_total = st->bytes_payload_padded + st->bytes_bitmap + st->bytes_offsets;
     st->pmr = 0.5 * (double)h.nnz / (double)(st->bytes_bitmap + st->bytes_offsets);
     st->fill = (double)Q * (double)h.sum_P / ((double)h.M * (double)h.K);
@@ -297,11 +422,9 @@ void make_schedule(const HostMatrix& h, int n_cta, int G, std::vector<uint32_t>*
     // strip, so balancing bytes alone overloads the CTAs that get the sparse strips. Measured on a
     // row-varying 4096 x 11008 matrix with sorted rows: N = 8 11.5 -> 10.0 us, N = 32 25.5 -> 20.3 us
     // with cost = bytes + 2 x the average tile; uniform matrices are unaffected.
-    // (US_BALANCE: 0 = bytes only, 1 = tiles only, k >= 2 = bytes + k x average tile)
-    static const int mode = [] { const char* e = std::getenv("US_BALANCE"); return e ? std::atoi(e) : 2; }();
     const uint64_t avg16 = std::max<uint64_t>(1, h.item_off[h.n_items] / (uint64_t)std::max<int64_t>(1, h.n_items));
     auto tile_cost = [&](uint32_t units16) -> uint64_t {
-        return mode == 0 ? units16 : mode == 1 ? avg16 : units16 + (uint64_t)mode * avg16;
+        return units16 + 2 * avg16;
     };
     std::vector<uint64_t> prefix((size_t)h.n_items + 1, 0);
     std::vector<int32_t> strip_of((size_t)h.n_items), kr_of((size_t)h.n_items);
@@ -322,9 +445,7 @@ void make_schedule(const HostMatrix& h, int n_cta, int G, std::vector<uint32_t>*
     // finer byte balance of cutting inside strips (measured at N = 8: 11008 x 4096 11.2 -> 9.0 us,
     // 13824 x 5120 13.4 -> 11.2 us, 28672 x 8192 26.6 -> 25.0 us). With several K ranges every strip
     // goes through the workspace anyway and aligned cuts make no measurable difference.
-    static const int align_mode = [] { const char* e = std::getenv("US_STRIP_CUTS"); return e ? std::atoi(e) : 1; }();
-    // 0: only small matrices in one K range (< 4 strips per CTA); 1: always with one K range; 2: always
-    const bool whole_strips = align_mode >= 2 || (n_kr == 1 && (align_mode == 1 || h.n_strips < (int64_t)4 * n_cta));
+    const bool whole_strips = n_kr == 1;
     const int64_t g_last = h.n_segs - (n_kr - 1) * G;
     int64_t pos = 0;
     // Tilt (per mille): CTA 0 gets that much more than the average share, the last CTA that much less,
@@ -332,7 +453,7 @@ void make_schedule(const HostMatrix& h, int n_cta, int G, std::vector<uint32_t>*
     // launch (they land on the SMs whose tile copies take longest); 3 % of tilt takes 2 % off the
     // 28672 x 8192 case (25.0 -> 24.5 us), 6 % and more start to hurt other shapes, a negative tilt
     // costs 2 %.
-    static const int tilt = [] { const char* e = std::getenv("US_TILT"); return e ? std::atoi(e) : 30; }();
+    constexpr int tilt = 30;
     for (int c = 0; c <= n_cta; ++c) {
         // (only where a CTA's share is many strips: on small shares the rounding to strips decides)
         const double x = (double)c / (double)n_cta, a = (whole_strips && h.n_strips >= (int64_t)8 * n_cta) ? tilt * 1e-3 : 0.0;
@@ -352,10 +473,9 @@ void make_schedule(const HostMatrix& h, int n_cta, int G, std::vector<uint32_t>*
     // restaging of X behind a CTA-wide barrier (about 9 K cycles), and the whole launch waits for
     // those few CTAs. Give every range a whole number of CTAs in proportion to its bytes and split
     // each range evenly among its own.
-    static const int range_mode = [] { const char* e = std::getenv("US_RANGE_CTAS"); return e ? std::atoi(e) : 1; }();
     // (Not with one-segment ranges -- the direct mode: there a range is small, changing it is cheap,
     // and rounding CTAs to many ranges unbalances them: N = 64 on 28672 x 8192 87 -> 93 us.)
-    if (range_mode && n_kr > 1 && G > 1 && n_kr * 8 <= n_cta) {
+    if (n_kr > 1 && G > 1 && n_kr * 8 <= n_cta) {
         std::vector<int64_t> r_beg((size_t)n_kr + 1, 0);
         for (int64_t kr = 0; kr < n_kr; ++kr) r_beg[kr + 1] = std::min<int64_t>(h.n_items, (kr + 1) * h.n_strips * G);
         r_beg[n_kr] = h.n_items;

@@ -16,6 +16,9 @@
 //                 stream in words; shorter streams are zero padded. Word (j, l) of either
 //                 matrix sits in shared-memory bank l: every decode load is conflict free.
 //   * per-tile offsets: item_off[t] in units of 16 bytes, n_items + 1 entries.
+//
+// Any other valid IE-BME format (other H_L, R_A, C_A, narrow tiles) is encoded on the host in the
+// paper's own array layout (GenericArrays) for us_get_stats / us_decode; no kernel reads it.
 #pragma once
 #include <cstdint>
 #include <vector>
@@ -24,9 +27,20 @@
 
 namespace us {
 
+// The paper's three arrays for an arbitrary (H_L, K_L, R_A, C_A) (Sec. V-A "Storage Arrays"): what
+// a format without a kernel is encoded into, for us_get_stats / us_decode.
+struct GenericArrays {
+    int64_t n_lt = 0, words_per_lt = 0;
+    std::vector<uint64_t> bitmaps;   // Union Bitmaps: row-major, leftmost column = LSB, 64-bit words
+    std::vector<uint32_t> offsets;   // Union Value Offsets, in INT4 values, n_lt + 1 entries
+    std::vector<uint8_t> values;     // Compressed Values: two per byte, even index in the low nibble
+};
+
 struct HostMatrix {
     int64_t M = 0, K = 0, Mp = 0, Kp = 0;
     us_format fmt{16, 1024, 2, 1};
+    bool kernel_layout = true;   // false: generic arrays only (host-only formats)
+    GenericArrays gen;
     int32_t nkb = 0;        // k-blocks (32 columns) per tile
     int32_t mask_rows = 0;  // nkb / 4
     int64_t n_strips = 0, n_segs = 0, n_items = 0;
@@ -51,6 +65,6 @@ void make_schedule(const HostMatrix& h, int n_cta, int G, std::vector<uint32_t>*
                    int* max_local_strips);
 
 // Default K_L for a shape when the caller passes no format.
-int32_t default_K_L(int64_t M, int64_t K);
+int32_t default_K_L(int64_t M, int64_t K, int n_sm);
 
 }  // namespace us

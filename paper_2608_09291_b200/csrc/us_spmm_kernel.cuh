@@ -56,10 +56,12 @@ struct SpmmParams {
                                                 // segment count, n_strips * G
     int32_t s_local;            // local mode: strips a CTA may hold in shared memory (0 = direct mode)
     int32_t lut_rep;            // copies of the selector table in shared memory (8 or 32)
-    int32_t nkb, mask_rows, K_L;
+    int32_t mask_rows, K_L;
     uint32_t slot_bytes;        // ring slot size (max tile blob + slack), multiple of 128
     int32_t x_fast;             // 2: K % 32 == 0 (16-byte loads); 1: K % 8 == 0 (4-byte loads); 0: bytes
     int32_t fp16_out;
+    uint32_t wait_ns_hi;        // bounded waits give up after this many ns >> 10
+    uint32_t withhold;          // test hook: position whose copy is never issued (~0u = none)
     // CTA c owns positions [cta_begin[c], cta_begin[c+1]) of the (K range, strip, segment) order.
     // Kept in the kernel parameters: the schedule is known without a global-memory round trip.
     uint32_t cta_begin[kMaxCtas + 1];
@@ -137,22 +139,46 @@ __device__ __forceinline__ uint64_t global_timer_ns()
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait: gives up after ~2 s of wall time (or 2^22 polls) instead of spinning forever.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+// The same with a suspend-time hint: the thread sleeps in hardware (taking no issue slots from the
+// decoding warps) until the phase completes or about `ns` nanoseconds have passed.
+__device__ __forceinline__ bool mbar_try_wait_sleep(uint32_t bar, uint32_t parity, uint32_t ns)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(ns)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after limit_hi << 10 ns of wall time (~2 s unless a test shortens it)
+// instead of spinning forever. Between checks of the clock the thread sleeps on the barrier.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit_hi)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_timer_ns();
+    const uint32_t nap = limit_hi < 64u ? 1000u : 20000u;   // ns per sleep
     for (uint32_t it = 0; it < (1u << 22); ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (global_timer_ns() - t0 > 2000000000ull) break;
+        if (mbar_try_wait_sleep(bar, parity, nap)) return true;
+        if (((global_timer_ns() - t0) >> 10) > limit_hi) break;
     }
     return false;
 }
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
+// The weights are read once per call: their lines are marked evict-first in L2, so that they do not
+// push out what is reused (the activations every CTA reads, the split-K workspace).
+__device__ __forceinline__ uint64_t l2_evict_first_policy()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy)
 {
     asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy)
         : "memory");
 }
 __device__ __forceinline__ void mma_s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
@@ -354,16 +380,14 @@ __device__ __forceinline__ void store_rows(const StoreCtx p, const int (&v)[NT][
 // issued before any is used. Block i takes its first four fragment bytes from the window that
 // STARTS at pos[i] and its last four from the window that ENDS at pos[i+1]; the window at
 // pos[4] is carried to the next word, so each word is self-contained (no peeled first or last).
-// CH independent chains walk consecutive ranges of the tile's mask words.
 // All addresses are 32-bit shared-memory addresses: slot_a = the staged tile, lut_a = selector
 // table + 4*lane, xb_a = this lane's first B-fragment of the tile's segment.
 // XP: X is staged packed (one word per lane, k-block and n-tile) instead of as int8 (two words).
-template <int NT, int CH, bool XP>
+template <int NT, bool XP>
 __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, uint32_t lut_stride,
                                              uint32_t xb_a, int xstride, int mask_rows, int lane,
                                              int (&c)[NT][4])
 {
-    const int rows_per = mask_rows / CH;
     const uint32_t mask_a = slot_a + 4u * lane;
     const uint32_t pay_a = slot_a + 128u * mask_rows + 4u * lane;
     constexpr bool kPreX = NT <= 2;   // small N: fetch the X fragments together with the windows
@@ -375,72 +399,49 @@ __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, ui
         }
         return lds64(a);
     };
-    uint32_t b8[CH];       // 8 * (byte position in the lane's payload stream), per chain
-    uint32_t cw0[CH], cw1[CH];   // carried window: the two words at / after the chain's position
-    b8[0] = 0;
+    uint32_t b8 = 0;                                     // 8 * (byte position in the lane's payload stream)
+    uint32_t cw0 = lds32_at<0>(pay_a), cw1 = lds32_at<128>(pay_a);   // carried window: the words at / after the position
+    for (int w = 0; w < mask_rows; ++w) {
+        uint32_t pos[5], wm1[4], w0[4], w1[4], e[4];
+        uint2 xf[4][kPreX ? NT : 1];
+        const uint32_t mw = lds32(mask_a + 128u * w);
+        pos[0] = b8;
 #pragma unroll
-    for (int ch = 1; ch < CH; ++ch) {
-        uint32_t n = 0;
-        for (int w = 0; w < rows_per; ++w) n += (uint32_t)__popc(lds32(mask_a + 128u * ((ch - 1) * rows_per + w)));
-        b8[ch] = b8[ch - 1] + 8u * n;
-    }
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t cum = (i == 3) ? mw : (mw & ((1u << (8 * i + 8)) - 1u));
+            pos[i + 1] = b8 + 8u * (uint32_t)__popc(cum);
+            e[i] = lut_a + prmt(mw, 0u, 0x4440u + i) * lut_stride;   // address of the table entry
+        }
+        b8 = pos[4];
 #pragma unroll
-    for (int ch = 0; ch < CH; ++ch) {
-        const uint32_t a = pay_a + ((b8[ch] >> 5) << 7);
-        cw0[ch] = lds32_at<0>(a);
-        cw1[ch] = lds32_at<128>(a);
-    }
-    for (int w = 0; w < rows_per; ++w) {
-        uint32_t pos[CH][5], wm1[CH][4], w0[CH][4], w1[CH][4], e[CH][4];
-        uint2 xf[CH][4][kPreX ? NT : 1];
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t a = pay_a + ((pos[i + 1] >> 5) << 7);   // window at the block's END
+            wm1[i] = lds32_at<-128>(a);
+            w0[i] = lds32_at<0>(a);
+            w1[i] = lds32_at<128>(a);
+            e[i] = lds32(e[i]);
+            if (kPreX) {
 #pragma unroll
-        for (int ch = 0; ch < CH; ++ch) {
-            const uint32_t mw = lds32(mask_a + 128u * (ch * rows_per + w));
-            pos[ch][0] = b8[ch];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const uint32_t cum = (i == 3) ? mw : (mw & ((1u << (8 * i + 8)) - 1u));
-                pos[ch][i + 1] = b8[ch] + 8u * (uint32_t)__popc(cum);
-                e[ch][i] = lut_a + prmt(mw, 0u, 0x4440u + i) * lut_stride;   // address of the table entry
+                for (int nt = 0; nt < NT; ++nt) xf[i][nt] = ldx(xb_a + kXStep * (4 * w + i) + nt * 8 * xstride);
             }
-            b8[ch] = pos[ch][4];
         }
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
+        for (int i = 0; i < 4; ++i) {
+            // first four bytes: the window starting at pos[i] (carried, or the previous block's)
+            const uint32_t s0 = (i == 0) ? cw0 : w0[i - 1];
+            const uint32_t s1 = (i == 0) ? cw1 : w1[i - 1];
+            const uint32_t lo = __funnelshift_r(s0, s1, pos[i]);
+            const uint32_t prev = __funnelshift_r(wm1[i], w0[i], pos[i + 1]);
+            const uint32_t d0 = prmt(lo, kFill, e[i]);
+            const uint32_t d1 = prmt(prev, kFill, e[i] >> 16);
+            const uint32_t e0 = d0 & 0x0F0F0F0Fu, e1 = d1 & 0x0F0F0F0Fu;
 #pragma unroll
-            for (int ch = 0; ch < CH; ++ch) {
-                const uint32_t a = pay_a + ((pos[ch][i + 1] >> 5) << 7);   // window at the block's END
-                wm1[ch][i] = lds32_at<-128>(a);
-                w0[ch][i] = lds32_at<0>(a);
-                w1[ch][i] = lds32_at<128>(a);
-                e[ch][i] = lds32(e[ch][i]);
-                if (kPreX) {
-#pragma unroll
-                    for (int nt = 0; nt < NT; ++nt)
-                        xf[ch][i][nt] = ldx(xb_a + kXStep * (4 * (ch * rows_per + w) + i) + nt * 8 * xstride);
-                }
+            for (int nt = 0; nt < NT; ++nt) {
+                const uint2 b = kPreX ? xf[i][nt] : ldx(xb_a + kXStep * (4 * w + i) + nt * 8 * xstride);
+                mma_s8(c[nt], d0, e0, d1, e1, b.x, b.y);
             }
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-#pragma unroll
-            for (int ch = 0; ch < CH; ++ch) {
-                // first four bytes: the window starting at pos[i] (carried, or the previous block's)
-                const uint32_t s0 = (i == 0) ? cw0[ch] : w0[ch][i - 1];
-                const uint32_t s1 = (i == 0) ? cw1[ch] : w1[ch][i - 1];
-                const uint32_t lo = __funnelshift_r(s0, s1, pos[ch][i]);
-                const uint32_t prev = __funnelshift_r(wm1[ch][i], w0[ch][i], pos[ch][i + 1]);
-                const uint32_t d0 = prmt(lo, kFill, e[ch][i]);
-                const uint32_t d1 = prmt(prev, kFill, e[ch][i] >> 16);
-                const uint32_t e0 = d0 & 0x0F0F0F0Fu, e1 = d1 & 0x0F0F0F0Fu;
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
-                    const uint2 b = kPreX ? xf[ch][i][nt]
-                                          : ldx(xb_a + kXStep * (4 * (ch * rows_per + w) + i) + nt * 8 * xstride);
-                    mma_s8(c[nt], d0, e0, d1, e1, b.x, b.y);
-                }
-            }
-#pragma unroll
-        for (int ch = 0; ch < CH; ++ch) { cw0[ch] = w0[ch][3]; cw1[ch] = w1[ch][3]; }
+        }
+        cw0 = w0[3]; cw1 = w1[3];
     }
 }
 
@@ -469,6 +470,14 @@ __device__ __forceinline__ uint32_t fdiv(uint32_t u, unsigned long long m)
 {
     return (uint32_t)(((unsigned long long)u * m) >> 40);
 }
+
+// Stage-timer buffer (unsigned long long words), written by the TIMED build: one record of kWarpRec
+// words per (CTA, warp) -- [0] valid, [1] wait, [2] decode, [3] epilogue, [4] lifetime, [5] cycles
+// before the first tile, [6] start ns, [7] activations staged ns, [8] end ns, [9..12] prologue
+// checkpoints (cycles: range known, copies issued, table done, X staged), [13] ns past the
+// dependency wait.
+constexpr int kWarpRec = 16, kMaxWarpsPerCta = 16;
+constexpr int kTimerWords = kWarpRec * kMaxWarpsPerCta * kMaxCtas;
 
 // LA = local mode (shared-memory strip accumulators), else direct mode.
 // TIMED = record the diagnostic stage timers (a separate instantiation, so that the production
@@ -501,13 +510,12 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
     uint8_t* my_ring = ring0 + (size_t)warp * STAGES * p.slot_bytes;
 
     const uint32_t beg = p.cta_begin[blockIdx.x], end = p.cta_begin[blockIdx.x + 1];
+    const uint64_t w_policy = l2_evict_first_policy();
     // Programmatic dependent launch: let the next kernel of the stream start its own prologue
     // (parameter fetch, offsets, first weight tiles) while this one is still working.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (beg >= end) return;
-#ifndef US_EXP_EPI_TIMERS
     if (timing) dbg[0] = clock64() - t_start;
-#endif
 
     // position u of the processing order -> K range, strip, segment within the range, tile index
     const uint32_t kr_stride = (uint32_t)p.n_strips * (uint32_t)p.G;
@@ -611,29 +619,27 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
             const uint32_t u = static_pos(s);
             if (s < STAGES) {
                 item[s] = u;
-                if (u < end && lane == 0) {
+                if (u < end && lane == 0 && u != p.withhold) {
                     const uint32_t bar = smem_u32(&bars[warp * STAGES + s]);
                     mbar_expect_tx(bar, (b - a) * 16u);
-                    bulk_g2s(smem_u32(my_ring + (size_t)s * p.slot_bytes), p.blob + (size_t)a * 16u, (b - a) * 16u, bar);
+                    bulk_g2s(smem_u32(my_ring + (size_t)s * p.slot_bytes), p.blob + (size_t)a * 16u, (b - a) * 16u, bar, w_policy);
                 }
             } else {
                 ahead = u; po0 = a; po1 = b;
             }
         }
     }
-#ifndef US_EXP_EPI_TIMERS
     if (timing) dbg[1] = clock64() - t_start;
-#endif
     if (threadIdx.x == 0) *claim = beg + (uint32_t)n_static * (uint32_t)n_warps * R;
     // refill slot s with the position fetched ahead
     auto refill = [&](int s) {
-        if (lane == 0 && ahead < end) {
+        if (lane == 0 && ahead < end && ahead != p.withhold) {
             const uint32_t bytes = (po1 - po0) * 16u;
             const uint32_t bar = smem_u32(&bars[warp * STAGES + s]);
             // the warp's earlier generic-proxy reads of this slot are ordered before the refill
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             mbar_expect_tx(bar, bytes);
-            bulk_g2s(smem_u32(my_ring + (size_t)s * p.slot_bytes), p.blob + (size_t)po0 * 16u, bytes, bar);
+            bulk_g2s(smem_u32(my_ring + (size_t)s * p.slot_bytes), p.blob + (size_t)po0 * 16u, bytes, bar, w_policy);
         }
         return ahead;
     };
@@ -680,6 +686,8 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
     for (int i = threadIdx.x, sh = 31 - __clz(p.lut_rep); i < 256 * p.lut_rep; i += blockDim.x) lut[i] = lut1[i >> sh];
 
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    const unsigned long long g_wait = timing ? global_timer_ns() : 0;
+    unsigned long long g_x = 0;
     // The activations of the CTA's first K range: fetch them into registers now, ahead of the
     // staging pass; and the activation scales of this lane's tokens.
     if (kPreScales && ScalePre<NT>::kSx && p.fp16_out) {
@@ -807,15 +815,11 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
         }
         __syncthreads();
     };
-#ifndef US_EXP_EPI_TIMERS
     if (timing) dbg[2] = clock64() - t_start;
-#endif
     // The first range is staged here, outside the loop, so that the prefetched X registers are
     // dead before the decode loop starts.
     stage_range(kr_first, g_first, true);
-#ifndef US_EXP_EPI_TIMERS
-    if (timing) dbg[3] = clock64() - t_start;
-#endif
+    if (timing) { dbg[3] = clock64() - t_start; g_x = global_timer_ns(); }
 
     for (int kr = kr_first; kr <= kr_last; ++kr) {
         const int g_kr = (kr == n_kr - 1) ? g_last : p.G;
@@ -838,7 +842,7 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
             if (u >= hi) break;
             const long long t0 = timing ? clock64() : 0;
             const uint32_t bar = smem_u32(&bars[warp * STAGES + cur]);
-            if (!mbar_wait_bounded(bar, (phase >> cur) & 1u)) {
+            if (!mbar_wait_bounded(bar, (phase >> cur) & 1u, p.wait_ns_hi)) {
                 if (lane == 0) atomicExch(p.err, kErrTimeout);
                 dead = true;
                 break;
@@ -864,13 +868,10 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
             const uint32_t slot_a = smem_u32(my_ring + (size_t)cur * p.slot_bytes);
             const uint32_t xb_a = XP ? smem_u32(x8) + (lane >> 2) * xstride + 4 * (lane & 3) + sgl * (p.K_L / 2)
                                      : smem_u32(x8) + (lane >> 2) * xstride + 8 * (lane & 3) + sgl * p.K_L;
-            process_tile<NT, 1, XP>(slot_a, lut_a, 4u * (uint32_t)p.lut_rep, xb_a, xstride, p.mask_rows, lane, c);
+            process_tile<NT, XP>(slot_a, lut_a, 4u * (uint32_t)p.lut_rep, xb_a, xstride, p.mask_rows, lane, c);
             __syncwarp();
             const long long t2c = timing ? clock64() : 0;
 
-#ifdef US_EXP_EPI_TIMERS
-            long long te0 = clock64();
-#endif
             // refill this slot right away, so that the copy overlaps the bookkeeping
             {
                 const uint32_t issued = refill(cur);
@@ -880,9 +881,6 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
             }
             cur = (cur + 1 == STAGES) ? 0 : cur + 1;
 
-#ifdef US_EXP_EPI_TIMERS
-            long long te1 = clock64(); dbg[0] += te1 - te0;
-#endif
             // ---- fragment sums -> partial Y of this tile, added to the run's sums ----
             const int32_t* sxp = sx16 + sgl * (NT * 8);
 #pragma unroll
@@ -901,9 +899,6 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
             for (int s = 0; s < STAGES; ++s)
                 if (s == cur) u_next = item[s];
             const bool more = (u_next == u + 1u) && (u_next < hi) && (sgl + 1 < g_kr);
-#ifdef US_EXP_EPI_TIMERS
-            long long te2 = clock64(); dbg[1] += te2 - te1;
-#endif
             if (!more) {
                 // what happens to the run's sums: 0 = nothing more, 1 = store (the strip is complete
                 // here), 2 = add to the global workspace and announce `tell` tiles
@@ -955,13 +950,7 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
                 for (int nt = 0; nt < NT; ++nt) y[nt][0] = y[nt][1] = y[nt][2] = y[nt][3] = 0;
                 y_n = 0;
             }
-#ifdef US_EXP_EPI_TIMERS
-            long long te3 = clock64(); dbg[2] += te3 - te2;
-#endif
             fetch_ahead();
-#ifdef US_EXP_EPI_TIMERS
-            dbg[3] += clock64() - te3;
-#endif
             if (timing) {
                 const long long t3 = clock64();
                 t_wait += t1 - t0; t_decode += t2c - t1; t_epi += t3 - t2c;
@@ -975,29 +964,22 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
     if (dead) {
 #pragma unroll
         for (int s = 0; s < STAGES; ++s) {
-            if (item[s] < end) {
+            if (item[s] < end && item[s] != p.withhold) {
                 const uint32_t bar = smem_u32(&bars[warp * STAGES + s]);
-                if (!mbar_wait_bounded(bar, (phase >> s) & 1u) && lane == 0) atomicExch(p.err, kErrTimeout);
+                if (!mbar_wait_bounded(bar, (phase >> s) & 1u, p.wait_ns_hi) && lane == 0) atomicExch(p.err, kErrTimeout);
             }
         }
     }
     if (timing && lane == 0) {
-        const long long t_end = clock64();
-        atomicAdd(p.timers + 0, (unsigned long long)t_wait);
-        atomicAdd(p.timers + 1, (unsigned long long)t_decode);
-        atomicAdd(p.timers + 2, (unsigned long long)t_epi);
-        atomicAdd(p.timers + 3, (unsigned long long)(t_end - t_start));
-        atomicAdd(p.timers + 4, 1ull);
-        atomicAdd(p.timers + 5, (unsigned long long)(t_first - t_start));
-        atomicMax(p.timers + 6, (unsigned long long)(t_end - t_start));
-        atomicMin(p.timers + 7, g_start);
-        atomicMax(p.timers + 8, (unsigned long long)global_timer_ns());
-        for (int i = 0; i < 4; ++i) atomicAdd(p.timers + 9 + i, (unsigned long long)dbg[i]);
-        // per-CTA sums: warp lifetimes, waits, decode; and the CTA's start offset from the first one
-        atomicAdd(p.timers + 16 + 4 * blockIdx.x + 0, (unsigned long long)(t_end - t_start));
-        atomicAdd(p.timers + 16 + 4 * blockIdx.x + 1, (unsigned long long)t_wait);
-        atomicAdd(p.timers + 16 + 4 * blockIdx.x + 2, (unsigned long long)t_decode);
-        if (warp == 0) p.timers[16 + 4 * blockIdx.x + 3] = g_start;
+        // one record per warp, plain stores (contended atomics here would hold up the warps still
+        // decoding: global and shared-memory instructions share the SM's memory pipeline)
+        unsigned long long* R = p.timers + (size_t)kWarpRec * ((size_t)blockIdx.x * kMaxWarpsPerCta + (size_t)warp);
+        R[1] = (unsigned long long)t_wait; R[2] = (unsigned long long)t_decode; R[3] = (unsigned long long)t_epi;
+        R[4] = (unsigned long long)(clock64() - t_start); R[5] = (unsigned long long)(t_first - t_start);
+        R[6] = g_start; R[7] = g_x; R[8] = (unsigned long long)global_timer_ns();
+        R[9] = (unsigned long long)dbg[0]; R[10] = (unsigned long long)dbg[1]; R[11] = (unsigned long long)dbg[2];
+        R[12] = (unsigned long long)dbg[3]; R[13] = g_wait;
+        R[0] = 1ull;
     }
 }
 
