@@ -2,12 +2,19 @@
 """Benchmark of the W4A4 bitmap-sparse SpMM (one JSON line on stdout).
 
 Workload of the headline line: LLaMA-2-7B-shaped attention projections, W 4096x4096 INT4 at 50 %
-uniform sparsity, X 4096xN INT4 with N = 8, fused fp16 dequant output. One step = one SpMM on each
+uniform sparsity, X 4096xN INT4 with N = 8, fused fp16 dequant output. One pass = one SpMM on each
 of R distinct encoded weight buffers (R * bytes > 3x the L2 size, so every launch streams its
-weights from HBM). The sweep over sparsity {30, 50, 70 %} x N {1, 8, 16, 32} and the 70B-shaped
-FFN (28672x8192, 60 %) N sweep are reported in the same line under "sweep".
+weights from HBM); one step = as many passes as make the timed region at least half a second. The
+other configurations (1024x1024; sparsity {30, 50, 70 %} x N {1, 8, 16, 32}; the 7B-shaped FFN with
+row-varying density; the 13B-shaped decoder layer; the 70B-shaped FFN N sweep) are reported in the
+same line under "sweep".
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-sweep]
+  python bench.py --only M,K,s,N[,int32|fp16[,K_L[,N_max]]]     one case with the kernel's stage
+                                                               timers (the command of the ncu captures)
+
+With --gpus N > 1 and no torchrun environment the script starts itself N times under
+torch.distributed.run (one replica per GPU, no data-path collective).
 """
 from __future__ import annotations
 
@@ -28,17 +35,40 @@ if str(ROOT) not in sys.path:
 METRIC = "w4a4_spmm_achieved_hbm_gbs"
 UNIT = "GB/s"
 HEAD = dict(M=4096, K=4096, s=0.5, N=8, seed=201)
+WORKLOAD = ("llama2-7b attention projection 4096x4096 INT4, 50% uniform sparsity, N=8, fused fp16 dequant; "
+            "bytes counted at local tiles of 16x512, one union-mask bit per 2x1 values")
+HEAD_K_L = 512                       # tile width the byte count of both arms refers to
 CONTRACT_PEAK_GBS = 8000.0
 L2_BYTES_FALLBACK = 126 * 1024 * 1024
+MIN_TIMED_SECONDS = 0.5
+
+
+def io_bytes(M: int, K: int, N: int, fp16: bool) -> int:
+    """X, Y and (fp16 output) the two scale vectors."""
+    return N * ((K + 1) // 2) + N * M * (2 if fp16 else 4) + (2 * (M + N) if fp16 else 0)
 
 
 def algorithmic_bytes(stats: dict, N: int, fp16: bool) -> int:
     """What the method must move once per call: packed INT4 values of the active union-mask
     positions, union bitmaps, per-tile offsets, X, Y and (fp16 output) the two scale vectors.
     Padding of the stored payload is NOT counted: it shows up as traffic above this figure."""
-    M, K = stats["M"], stats["K"]
     w = stats["bytes_payload"] + stats["bytes_bitmap"] + stats["bytes_offsets"]
-    return w + N * ((K + 1) // 2) + N * M * (2 if fp16 else 4) + (2 * (M + N) if fp16 else 0)
+    return w + io_bytes(stats["M"], stats["K"], N, fp16)
+
+
+def bytes_q1(stats: dict, N: int, fp16: bool) -> int:
+    """The same call with a per-element bitmap (one bit per weight, 16x64 local tiles): only the
+    true nonzeros are stored. Closed form from the handle's own nonzero count."""
+    M, K = stats["M"], stats["K"]
+    mp, kp = (M + 15) // 16 * 16, (K + 63) // 64 * 64
+    n_lt = (mp // 16) * (kp // 64)
+    return (stats["nnz"] + 1) // 2 + mp * kp // 8 + 4 * (n_lt + 1) + io_bytes(M, K, N, fp16)
+
+
+def bytes_dense_int4(stats: dict, N: int, fp16: bool) -> int:
+    """The same call on the dense INT4 weight (no bitmap, no pruning exploited)."""
+    M, K = stats["M"], stats["K"]
+    return (M * K + 1) // 2 + io_bytes(M, K, N, fp16)
 
 
 def measured_peaks():
@@ -115,7 +145,7 @@ def reference_arm(args, rank: int):
     W = workloads.make_weight(HEAD["M"], HEAD["K"], HEAD["s"], HEAD["seed"])
     X = workloads.make_x(HEAD["K"], 32, HEAD["seed"])[: HEAD["N"]]
     s_w, s_x = workloads.make_scales(HEAD["M"], 32, HEAD["seed"])
-    st = oracle.encode(W, 16, 512, 2, 1)["stats"]
+    st = oracle.encode(W, 16, HEAD_K_L, 2, 1)["stats"]
     stats = dict(M=HEAD["M"], K=HEAD["K"], bytes_payload=st["bytes_payload"],
                  bytes_bitmap=st["bytes_bitmap"], bytes_offsets=st["bytes_offsets"])
     per_call = algorithmic_bytes(stats, HEAD["N"], True)
@@ -139,8 +169,7 @@ def reference_arm(args, rank: int):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32",
         "data": "synthetic",
-        "config": {"workload": "llama2-7b attention projection 4096x4096 INT4, 50% sparsity, N=8, fp16 dequant",
-                   "flush": "n/a (CPU)"},
+        "config": {"workload": WORKLOAD, "flush": "n/a (CPU)"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -210,6 +239,26 @@ class Case:
             sw.check()
         return e0.elapsed_time(e1) * 1e-3 / (passes * len(self.sw))   # seconds per launch
 
+    def time_isolated(self, N, fp16, launches=40):
+        """One launch at a time: events around every single call with a synchronisation in between,
+        so that nothing of the next launch overlaps it (the pipelined figure of time_passes lets a
+        launch's prologue run under its predecessor). Median over the launches, in seconds."""
+        torch = self.torch
+        xs = self.sxd if fp16 else None
+        out = self.Y16 if fp16 else self.Y32
+        ts = []
+        for i in range(launches + 3):
+            sw = self.sw[i % len(self.sw)]
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            sw.spmm(self.Xd, N, xs, out=out[:N])
+            e1.record()
+            torch.cuda.synchronize()
+            if i >= 3:
+                ts.append(e0.elapsed_time(e1) * 1e-3)
+        return float(np.median(ts))
+
     def close(self):
         for sw in self.sw:
             sw.close()
@@ -245,14 +294,25 @@ def run_ours(args, rank: int, local_rank: int, world: int):
     W = workloads.make_weight(HEAD["M"], HEAD["K"], HEAD["s"], HEAD["seed"])
     Xall = workloads.make_x(HEAD["K"], 32, HEAD["seed"])
     s_w, s_x = workloads.make_scales(HEAD["M"], 32, HEAD["seed"])
-    probe = binding.us_encode(W, s_w, None, 32, binding.US_ENCODE_HOST_ONLY)
+    head_fmt = (16, HEAD_K_L, 2, 1)
+    probe = binding.us_encode(W, s_w, head_fmt, 32, binding.US_ENCODE_HOST_ONLY)
     pstats = binding.us_get_stats(probe)
     binding.us_destroy(probe)
     R = replicas_for(pstats, l2)
-    head = Case(binding, torch, W, s_w, Xall, s_x, 32, R)
+    head = Case(binding, torch, W, s_w, Xall, s_x, 32, R, fmt=head_fmt)
     N = HEAD["N"]
     alg = algorithmic_bytes(head.stats, N, True)
     g = head.graph(N, True)
+    # passes per step: the timed region (steps x passes x R launches) lasts at least half a second
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize()
+    t_probe = time.perf_counter()
+    for _ in range(10):
+        g.replay()
+    torch.cuda.synchronize()
+    t_pass = max(1e-6, (time.perf_counter() - t_probe) / 10)
+    passes = max(1, int(np.ceil(MIN_TIMED_SECONDS / (t_pass * max(1, args.steps)))))
 
     def barrier():
         if dist is not None:
@@ -260,14 +320,16 @@ def run_ours(args, rank: int, local_rank: int, world: int):
         torch.cuda.synchronize()
 
     for _ in range(max(args.warmup, 3)):
-        g.replay()
+        for _ in range(passes):
+            g.replay()
     barrier()
     sampler = ClockSampler(visible_device_index(local_rank))
     sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(args.steps):
-        g.replay()
+        for _ in range(passes):
+            g.replay()
     e1.record()
     sampler.sample()
     torch.cuda.synchronize()
@@ -276,9 +338,11 @@ def run_ours(args, rank: int, local_rank: int, world: int):
     for sw in head.sw:
         sw.check()
     dt = max_over_ranks(e0.elapsed_time(e1) * 1e-3, dist, "cuda")
-    launches = args.steps * R
+    launches = args.steps * passes * R
     per_launch = dt / launches
     value = alg * launches * world / dt / 1e9
+    t_iso = head.time_isolated(N, True)
+    q1, dn = bytes_q1(head.stats, N, True), bytes_dense_int4(head.stats, N, True)
 
     # ---- end to end: host buffers, H2D of X and scales, D2H of Y inside the timed region --------
     # One step = R SpMMs, each with its own (X | activation scales) block in pinned host memory and
@@ -361,17 +425,20 @@ def run_ours(args, rank: int, local_rank: int, world: int):
         "warmup": max(args.warmup, 3), "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
         "config": {
-            "workload": "llama2-7b attention projection 4096x4096 INT4, 50% uniform sparsity, N=8, "
-                        "fused fp16 dequant; one step = one SpMM on each of R distinct weight buffers",
-            "replicas_per_step": R, "format": list(head.stats["fmt"]),
+            "workload": WORKLOAD,
+            "step": f"{passes} passes of one SpMM on each of {R} distinct weight buffers",
+            "replicas_per_pass": R, "passes_per_step": passes, "format": list(head.stats["fmt"]),
             "flush": f"inputs larger than L2: {R} x {head.stats['bytes_total']} B of weights rotate "
                      f"through a {l2} B L2",
             "launch": "CUDA graph of one step, replayed",
             "parallelism": "replicas only" if world > 1 else "1 gpu",
         },
         "us_per_spmm": per_launch * 1e6,
+        "us_per_spmm_isolated": t_iso * 1e6,
         "dense_equiv_tops": 2.0 * HEAD["M"] * HEAD["K"] * N / per_launch / 1e12,
         "pct_of_8tbs": 100.0 * (alg / per_launch / 1e9) / CONTRACT_PEAK_GBS,
+        "bytes_q1": q1, "pct_of_8tbs_on_q1_bytes": 100.0 * (q1 / per_launch / 1e9) / CONTRACT_PEAK_GBS,
+        "bytes_dense_int4": dn, "us_dense_int4_at_8tbs": dn / CONTRACT_PEAK_GBS / 1e3,
         "clocks": clocks,
         "gpu_launches": launches,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -394,7 +461,7 @@ def run_ours(args, rank: int, local_rank: int, world: int):
             out["roofline_large"] = {"bound": "hbm", "achieved": r["gbs"], "peak": peak_gbs, "unit": "GB/s",
                                      "frac": r["gbs"] / peak_gbs, "pct_of_8tbs": r["pct_of_8tbs"],
                                      "us": r["us"], "algorithmic_bytes": r["alg_bytes"],
-                                     "traffic": 102_094_336,   # read 98.02 MB + written 4.08 MB: profiles/us_spmm_kernel_28672x8192_s60_n8_int32.md
+                                     "traffic": TRAFFIC_BYTES_PER_LAUNCH_LARGE,
                                      "kernel": r["kernel"] + " on 28672x8192 s=0.6 N=8 int32"}
     if rank == 0:
         out["cpu_baseline"] = cpu_baseline(W, Xall[:N], s_w, s_x[:N], pstats)
@@ -411,16 +478,16 @@ def kernel_label(binding, handle, N):
             f"{g['block'] // 32} warps, {g['smem_bytes']} B shared memory)")
 
 
-# Measured DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the
-# headline kernel, from the ncu capture summarised in
-# profiles/us_spmm_kernel_4096x4096_s50_n8_fp16.md (8.2007 MB read, 0 written).
-TRAFFIC_BYTES_PER_LAUNCH = 8_200_704
+# Measured DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch, from the ncu
+# captures of the same kernel build (one launch each; commands in the capture summaries).
+TRAFFIC_BYTES_PER_LAUNCH = 8_200_704          # 4096x4096, s = 0.5, N = 8, fp16: 8.2007 MB read, 0 written
+TRAFFIC_BYTES_PER_LAUNCH_LARGE = 102_094_336  # 28672x8192, s = 0.6, N = 8, int32: 98.02 MB read + 4.08 MB written
 
 
 def sweep(binding, torch, workloads, l2, peak_gbs):
     rows = []
 
-    def run_case(name, M, K, s, seed, Ns, fp16, row_varying=False, flags=0):
+    def run_case(name, M, K, s, seed, Ns, outs, row_varying=False, flags=0):
         W = workloads.make_weight(M, K, s, seed, row_varying)
         Nmax = max(Ns)
         X = workloads.make_x(K, Nmax, seed)
@@ -430,32 +497,40 @@ def sweep(binding, torch, workloads, l2, peak_gbs):
         binding.us_destroy(probe)
         R = replicas_for(st, l2)
         case = Case(binding, torch, W, s_w, X, s_x, Nmax, R, flags=flags)
-        for N in Ns:
-            passes = max(3, int(2e-2 / max(1e-6, 3e-6 * R)))
-            t = case.time_passes(N, fp16, passes=min(passes, 200), warmup=3)
-            alg = algorithmic_bytes(case.stats, N, fp16)
-            rows.append({"case": name, "M": M, "K": K, "sparsity": s, "N": N, "out": "fp16" if fp16 else "int32",
-                         "us": t * 1e6, "alg_bytes": alg, "stored_bytes": binding.us_spmm_bytes(case.sw[0].handle, N, fp16),
-                         "gbs": alg / t / 1e9, "pct_of_8tbs": 100 * alg / t / 1e9 / CONTRACT_PEAK_GBS,
-                         "frac_of_measured": alg / t / 1e9 / peak_gbs,
-                         "dense_equiv_tops": 2.0 * M * K * N / t / 1e12, "replicas": R,
-                         "pmr": case.stats["pmr"], "kernel": kernel_label(binding, case.sw[0].handle, N)})
+        for fp16 in outs:
+            for N in Ns:
+                passes = max(3, int(2e-2 / max(1e-6, 3e-6 * R)))
+                t = case.time_passes(N, fp16, passes=min(passes, 200), warmup=3)
+                t_iso = case.time_isolated(N, fp16, launches=20)
+                alg = algorithmic_bytes(case.stats, N, fp16)
+                q1, dn = bytes_q1(case.stats, N, fp16), bytes_dense_int4(case.stats, N, fp16)
+                rows.append({"case": name, "M": M, "K": K, "sparsity": s, "N": N, "out": "fp16" if fp16 else "int32",
+                             "us": t * 1e6, "us_isolated": t_iso * 1e6, "alg_bytes": alg,
+                             "stored_bytes": binding.us_spmm_bytes(case.sw[0].handle, N, fp16),
+                             "gbs": alg / t / 1e9, "pct_of_8tbs": 100 * alg / t / 1e9 / CONTRACT_PEAK_GBS,
+                             "frac_of_measured": alg / t / 1e9 / peak_gbs,
+                             "bytes_q1": q1, "pct_of_8tbs_on_q1_bytes": 100 * q1 / t / 1e9 / CONTRACT_PEAK_GBS,
+                             "bytes_dense_int4": dn, "us_dense_int4_at_8tbs": dn / CONTRACT_PEAK_GBS / 1e3,
+                             "dense_equiv_tops": 2.0 * M * K * N / t / 1e12, "replicas": R,
+                             "pmr": case.stats["pmr"], "kernel": kernel_label(binding, case.sw[0].handle, N)})
         case.close()
         del case
         torch.cuda.empty_cache()
 
-    for i, s in enumerate((0.3, 0.5, 0.7)):
-        run_case("attn7b", 4096, 4096, s, 200 + i, [1, 8, 16, 32], True)
-    run_case("attn7b_qkv_fused", 12288, 4096, 0.5, 210, [8], True)   # Q, K, V stacked: one launch
-    run_case("ffn7b_up", 11008, 4096, 0.5, 300, [1, 8, 32], True, row_varying=True, flags=binding.US_ENCODE_SORT_ROWS)
-    run_case("ffn7b_up", 11008, 4096, 0.5, 300, [8], False, row_varying=True, flags=binding.US_ENCODE_SORT_ROWS)
-    run_case("ffn7b_down", 4096, 11008, 0.5, 302, [1, 8, 32], True, row_varying=True, flags=binding.US_ENCODE_SORT_ROWS)
-    run_case("ffn70b_up", 28672, 8192, 0.6, 500, [1, 4, 8, 16, 32, 64], False)
-    run_case("ffn70b_down", 8192, 28672, 0.6, 501, [1, 4, 8, 16, 32, 64], False)
+    SORT = binding.US_ENCODE_SORT_ROWS
+    run_case("single1024", 1024, 1024, 0.5, 0, [8], [False])                                  # config 1
+    for i, s in enumerate((0.3, 0.5, 0.7)):                                                    # config 2
+        run_case("attn7b", 4096, 4096, s, 200 + i, [1, 8, 16, 32], [True])
+    run_case("attn7b_qkv_fused", 12288, 4096, 0.5, 210, [8], [True])   # Q, K, V stacked: one launch
+    run_case("ffn7b_up", 11008, 4096, 0.5, 300, [1, 8, 32], [True, False], row_varying=True, flags=SORT)     # config 3
+    run_case("ffn7b_gate", 11008, 4096, 0.5, 301, [8], [True, False], row_varying=True, flags=SORT)
+    run_case("ffn7b_down", 4096, 11008, 0.5, 302, [1, 8, 32], [True, False], row_varying=True, flags=SORT)
+    run_case("ffn70b_up", 28672, 8192, 0.6, 500, [1, 4, 8, 16, 32, 64], [False])               # config 5
+    run_case("ffn70b_down", 8192, 28672, 0.6, 501, [1, 4, 8, 16, 32, 64], [False])
     # Bitmap-aware row pairing inside each strip (the per-strip form of Alg. 1): fewer union bits.
-    run_case("attn7b_paired", 4096, 4096, 0.5, 201, [8], True, flags=binding.US_ENCODE_PAIR_ROWS)
-    run_case("ffn70b_up_paired", 28672, 8192, 0.6, 500, [8], False, flags=binding.US_ENCODE_PAIR_ROWS)
-    for s in (0.3, 0.5, 0.7):
+    run_case("attn7b_paired", 4096, 4096, 0.5, 201, [8], [True], flags=binding.US_ENCODE_PAIR_ROWS)
+    run_case("ffn70b_up_paired", 28672, 8192, 0.6, 500, [8], [False], flags=binding.US_ENCODE_PAIR_ROWS)
+    for s in (0.3, 0.5, 0.7):                                                                  # config 4
         rows.append(layer_chain(binding, torch, workloads, l2, s))
     return rows
 
@@ -602,19 +677,35 @@ def run_only(args):
     case.close()
 
 
-def main():
+def torchrun_command(argv, gpus: int, port: int = 29541):
+    """The command that starts `gpus` replica processes of this script on one node."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(gpus),
+            "--master-addr", "127.0.0.1", "--master-port", str(port), str(Path(__file__).resolve())] + list(argv)
+
+
+def main(argv=None):
+    argv = list(sys.argv[1:] if argv is None else argv)
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--only", default=None, metavar="M,K,s,N[,int32|fp16[,K_L[,N_max]]]",
-                    help="time one case only (a few launches, no graph): the small run used for ncu captures")
-    args = ap.parse_args()
+                    help="time one case only, with the kernel's stage timers: the small run of the ncu captures")
+    args = ap.parse_args(argv)
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.gpus < 1:
+        ap.error("--gpus must be at least 1")
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1 and not args.only:
+        # replicas only: start one process per GPU (no data-path collective; the ranks meet for the
+        # barrier around the timed region and the maximum over ranks)
+        os.execvp(sys.executable, torchrun_command(argv, args.gpus))
+    if world != args.gpus and not args.only:
+        sys.exit(f"bench.py: --gpus {args.gpus} but WORLD_SIZE={world}: launch with "
+                 f"torch.distributed.run --nproc-per-node {args.gpus}, or without it")
     if args.impl == "reference":
         reference_arm(args, rank)
         return

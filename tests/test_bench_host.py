@@ -65,3 +65,26 @@ def test_reference_arm_prints_contract_line():
     assert d["impl"] == "reference" and d["metric"] == bench.METRIC and d["unit"] == bench.UNIT
     assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1
     assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["value"] > 0
+
+
+def test_gpus_flag_starts_replicas_or_refuses(monkeypatch):
+    """--gpus N outside a torchrun environment re-launches the script as N replica processes; inside
+    one, a world size that contradicts the flag is an error (the flag never lies about n_gpus)."""
+    cmd = bench.torchrun_command(["--gpus", "4", "--steps", "2"], 4, port=29999)
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"]
+    assert cmd[cmd.index("--nproc-per-node") + 1] == "4" and cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert cmd[-4:] == ["--gpus", "4", "--steps", "2"] and cmd[-5].endswith("bench.py")
+    called = {}
+    monkeypatch.delenv("WORLD_SIZE", raising=False)
+    monkeypatch.setattr(bench.os, "execvp", lambda exe, argv: called.setdefault("argv", argv) and (_ for _ in ()).throw(SystemExit(0)))
+    try:
+        bench.main(["--gpus", "2", "--steps", "1"])
+    except SystemExit:
+        pass
+    assert called["argv"][called["argv"].index("--nproc-per-node") + 1] == "2"
+    monkeypatch.setenv("WORLD_SIZE", "2")
+    try:
+        bench.main(["--gpus", "4"])
+        raise AssertionError("a contradicting world size must be refused")
+    except SystemExit as e:
+        assert "WORLD_SIZE=2" in str(e)

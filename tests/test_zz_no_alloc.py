@@ -4,10 +4,11 @@ trigger an allocator synchronisation, a program section where allocation calls a
 Its scratch is a fixed array inside the library instead of memory owned by the handle, so its
 results must be the very ones us_spmm gives -- checked here through the C ABI on two calls in a
 row (the array keeps the previous call's contents), in shapes that do send partial sums through the
-scratch. The file name keeps it last in collection order."""
+scratch, and against the CPU oracle as well. The file name keeps it last in collection order."""
 import numpy as np
 import pytest
 
+import oracle
 from paper_2608_09291_b200 import workloads
 
 pytestmark = pytest.mark.gpu
@@ -44,6 +45,7 @@ def test_matches_us_spmm_twice(b, M, K, N):
         b.us_spmm(h, Xd.data_ptr(), N, sxd.data_ptr(), ref16.data_ptr(), stream)
         torch.cuda.synchronize()
         assert b.us_last_error(h) == 0
+        exact = oracle.spmm_dense(W, X)
         for rep in range(2):
             got32 = torch.full((N, M), -7, dtype=torch.int32, device="cuda")
             got16 = torch.full((N, M), -7.0, dtype=torch.float16, device="cuda")
@@ -55,6 +57,9 @@ def test_matches_us_spmm_twice(b, M, K, N):
             # same kernel, same arithmetic: the fp16 outputs agree to the last bit, which is
             # inside the suite's fp16 bar (2e-3 relative or one ulp) with room to spare
             assert torch.equal(got16, ref16), f"call {rep}: fp16 output differs from us_spmm"
+            # and both are what the oracle says: INT32 bit for bit, fp16 within 2e-3 relative or one ulp
+            assert (got32.cpu().numpy() == exact).all(), f"call {rep}: INT32 output differs from the oracle"
+            assert oracle.fp16_within_tolerance(got16.cpu().numpy(), exact, s_w, s_x, rel=2e-3).all()
     finally:
         b.us_destroy(h)
 
