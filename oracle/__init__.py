@@ -13,6 +13,13 @@ What each function follows:
   lspd_idx_base        paper Sec. VI-B, idx_base(r, g)
   dequant              per-channel x per-token scaling to fp16; not in the paper -- defined by
                        the build's target: RN_fp16(double(acc) * double(s_w) * double(s_x))
+  absmax_f16           max |y| per token over a column range, exact in fp16
+  requant_int4         per-token symmetric INT4 re-quantisation of an fp16 activation. The paper
+                       takes INT4 activations as given (W4A4, Sec. VII-A) and defines no
+                       quantiser; the reading used here is the plain symmetric absmax one:
+                       s = max(RN_fp16(fp32(amax) / 7), 2^-24), code = clamp(RNE(fp32(y) /
+                       fp32(s)), -8, 7), division and rounding in fp32 (the kernel's precision:
+                       floating point decides an integer here, so both sides fix it)
 """
 from __future__ import annotations
 
@@ -178,6 +185,36 @@ def fp16_within_tolerance(got: np.ndarray, ref_acc: np.ndarray, s_w: np.ndarray,
     ulp = np.abs(np.spacing(ref16)).astype(np.float64)
     err = np.abs(got.astype(np.float64) - ref16.astype(np.float64))
     return err <= np.maximum(rel * np.abs(exact), ulp)
+
+
+def absmax_f16(y16: np.ndarray, m0: int = 0, m1: int | None = None) -> np.ndarray:
+    """amax[n] = max over m in [m0, m1) of |y16[n, m]| as fp16 (0 for an empty range)."""
+    y = np.asarray(y16, dtype=np.float16)[:, m0:m1]
+    if y.shape[1] == 0:
+        return np.zeros(y.shape[0], dtype=np.float16)
+    return np.abs(y).max(axis=1).astype(np.float16)
+
+
+FP16_TINY = np.float16(2.0 ** -24)   # the smallest positive fp16
+
+
+def requant_scale(amax16: np.ndarray) -> np.ndarray:
+    """s[n] = max(RN_fp16(fp32(amax[n]) / fp32(7)), 2^-24): the quantisation step per token."""
+    a = np.asarray(amax16, dtype=np.float16).astype(np.float32)
+    s = (a / np.float32(7.0)).astype(np.float16)
+    return np.maximum(s, FP16_TINY)
+
+
+def requant_int4(y16: np.ndarray, amax16: np.ndarray | None = None):
+    """(codes int8 (N, M) in [-8, 7], scales fp16 (N,)) of a finite fp16 activation y16 (N, M).
+    amax16 defaults to the per-token absmax over all of y16's columns."""
+    y = np.asarray(y16, dtype=np.float16)
+    if amax16 is None:
+        amax16 = absmax_f16(y)
+    s = requant_scale(amax16)
+    r = y.astype(np.float32) / s.astype(np.float32)[:, None]       # IEEE fp32 division
+    q = np.clip(np.rint(r), -8, 7).astype(np.int8)                  # rint: ties to even
+    return q, s
 
 
 def num_threads() -> int:
