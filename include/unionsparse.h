@@ -169,6 +169,40 @@ us_status us_spmm_static_scratch(us_handle* h, const void* X, int32_t N, const v
 us_status us_last_error(us_handle* h);
 
 /*
+ * Chained calls: fp16 activations in, INT4 inside, fp16 out.
+ *
+ * The paper evaluates the W4A4 kernel on INT4 activations that are given (Sec. VII-A) and defines
+ * no activation quantiser; these three calls have no counterpart in it. They let the output of one
+ * projection feed the next without a pass over the activations in between. The quantiser is the
+ * plain per-token symmetric one:
+ *     step[n] = max(RN_fp16(amax[n] / 7), 2^-24),  code = clamp(RNE(x / step[n]), -8, 7),
+ * amax[n] = max |x[n][k]| over the quantised columns, the quotients taken in IEEE fp32 (so the codes
+ * are reproducible bit for bit), and step[n] is the activation scale of the dequantisation.
+ *
+ * us_spmm_requant: Y16[n][m] = RN_fp16(sum_k W[m][k] * code(X16[n][k]) * w_scale[m] * step[n]).
+ *   X16     device, N rows of fp16, row n at X16 + n * ldx (elements), ldx >= K; finite values.
+ *           16-byte aligned rows (pointer and ldx % 8 == 0) take the vector path.
+ *   x_amax  device, N 32-bit words: the fp16 bit pattern of amax[n] (what us_absmax_f16 or an earlier
+ *           us_spmm_requant wrote).
+ *   Y16     device, N x M fp16 row-major. The handle must hold weight scales.
+ *   y_amax  device, N 32-bit words or NULL. If given, the call sets word n to the fp16 bit pattern of
+ *           max |Y16[n][m]| over amax_m0 <= m < amax_m1 (0 for an empty range): the x_amax of a next
+ *           call that reads columns [amax_m0, amax_m1) of Y16. It is cleared on the stream before the
+ *           kernel starts and must not be the x_amax of this same call.
+ * Everything else (stream order, workspace, errors, limits on N) is as for us_spmm.
+ *
+ * us_absmax_f16: amax[n] = max_k |X16[n][k]| for the head of a chain. N <= 65535.
+ * us_quantize_f16: the codes themselves, packed as us_spmm expects X (N x ceil(K/2) bytes, even k in
+ *   the low nibble), and the steps as fp16 bit patterns in x_scale (N entries, may be NULL).
+ * Both take device pointers, run on `stream`, keep no state and allocate nothing.
+ */
+us_status us_spmm_requant(us_handle* h, const void* X16, int64_t ldx, const void* x_amax, int32_t N,
+                          void* Y16, void* y_amax, int64_t amax_m0, int64_t amax_m1, void* stream);
+us_status us_absmax_f16(const void* X16, int64_t ldx, int32_t N, int64_t K, void* amax, void* stream);
+us_status us_quantize_f16(const void* X16, int64_t ldx, int32_t N, int64_t K, const void* amax, void* Xq,
+                          void* x_scale, void* stream);
+
+/*
  * Test hook for the bounded waits of the kernel (no counterpart in the paper): from now on every
  * us_spmm on this handle leaves out the copy of the tile at `position` of the processing order
  * (0 <= position < number of tiles) and gives up its waits after wait_us microseconds

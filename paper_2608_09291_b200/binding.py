@@ -23,6 +23,7 @@ US_ENCODE_SORT_ROWS = 2
 US_ENCODE_PAIR_ROWS = 4
 
 EXPORTS = ["us_encode", "us_get_stats", "us_decode", "us_get_row_order", "us_spmm", "us_spmm_static_scratch",
+           "us_spmm_requant", "us_absmax_f16", "us_quantize_f16",
            "us_last_error", "us_debug_withhold_copy", "us_stage_timers", "us_destroy", "us_spmm_bytes", "us_launch_info", "us_status_string"]
 
 
@@ -47,6 +48,10 @@ _lib.us_get_row_order.argtypes = [_vp, _vp]
 _lib.us_spmm.argtypes = [_vp, _vp, ctypes.c_int32, _vp, _vp, _vp]
 _lib.us_last_error.argtypes = [_vp]
 _lib.us_spmm_static_scratch.argtypes = [_vp, _vp, ctypes.c_int32, _vp, _vp, _vp]
+_lib.us_spmm_requant.argtypes = [_vp, _vp, ctypes.c_int64, _vp, ctypes.c_int32, _vp, _vp, ctypes.c_int64,
+                                 ctypes.c_int64, _vp]
+_lib.us_absmax_f16.argtypes = [_vp, ctypes.c_int64, ctypes.c_int32, ctypes.c_int64, _vp, _vp]
+_lib.us_quantize_f16.argtypes = [_vp, ctypes.c_int64, ctypes.c_int32, ctypes.c_int64, _vp, _vp, _vp, _vp]
 _lib.us_destroy.argtypes = [_vp]
 _lib.us_stage_timers.argtypes = [_vp, ctypes.c_int32, _vp, ctypes.c_int32]
 _lib.us_debug_withhold_copy.argtypes = [_vp, ctypes.c_int64, ctypes.c_int64]
@@ -131,6 +136,28 @@ def us_spmm_static_scratch(h: int, X_ptr: int, N: int, x_scale_ptr: int | None, 
            "us_spmm_static_scratch")
 
 
+def us_spmm_requant(h: int, X16_ptr: int, ldx: int, x_amax_ptr: int, N: int, Y16_ptr: int,
+                    y_amax_ptr: int | None = None, amax_m0: int = 0, amax_m1: int = 0,
+                    stream: int | None = None):
+    """Chained call: fp16 activations (row stride ldx elements) quantised per token to INT4 with
+    the step max|x| / 7 while they are staged, fp16 output, and optionally the per-token absmax
+    of output columns [amax_m0, amax_m1) for the next call. Device pointers as integers."""
+    _check(_lib.us_spmm_requant(h, X16_ptr, int(ldx), x_amax_ptr, int(N), Y16_ptr, y_amax_ptr,
+                                int(amax_m0), int(amax_m1), stream), "us_spmm_requant")
+
+
+def us_absmax_f16(X16_ptr: int, ldx: int, N: int, K: int, amax_ptr: int, stream: int | None = None):
+    """amax[n] (32-bit words holding fp16 bit patterns) = max_k |X16[n][k]|."""
+    _check(_lib.us_absmax_f16(X16_ptr, int(ldx), int(N), int(K), amax_ptr, stream), "us_absmax_f16")
+
+
+def us_quantize_f16(X16_ptr: int, ldx: int, N: int, K: int, amax_ptr: int, Xq_ptr: int,
+                    x_scale_ptr: int | None = None, stream: int | None = None):
+    """The INT4 codes of the chained call's quantiser, packed as us_spmm expects X, and the steps."""
+    _check(_lib.us_quantize_f16(X16_ptr, int(ldx), int(N), int(K), amax_ptr, Xq_ptr, x_scale_ptr, stream),
+           "us_quantize_f16")
+
+
 def us_last_error(h: int) -> int:
     return int(_lib.us_last_error(h))
 
@@ -185,6 +212,33 @@ def pack_int4(X: np.ndarray) -> np.ndarray:
     return np.ascontiguousarray(u[:, 0::2] | (u[:, 1::2] << 4))
 
 
+def absmax_f16(X16, out=None, stream=None):
+    """Per-token absmax of a device float16 (N, K) tensor or view (unit column stride), as the
+    int32 words the chained call takes."""
+    import torch
+    assert X16.dtype == torch.float16 and X16.stride(1) == 1
+    N, K = X16.shape
+    if out is None:
+        out = torch.empty(N, device=X16.device, dtype=torch.int32)
+    if stream is None:
+        stream = torch.cuda.current_stream(X16.device).cuda_stream
+    us_absmax_f16(X16.data_ptr(), X16.stride(0), N, K, out.data_ptr(), stream)
+    return out
+
+
+def quantize_f16(X16, amax, stream=None):
+    """(packed INT4 codes uint8 (N, ceil(K/2)), steps float16 (N,)) of a device float16 (N, K)."""
+    import torch
+    assert X16.dtype == torch.float16 and X16.stride(1) == 1
+    N, K = X16.shape
+    Xq = torch.empty((N, (K + 1) // 2), device=X16.device, dtype=torch.uint8)
+    sc = torch.empty(N, device=X16.device, dtype=torch.float16)
+    if stream is None:
+        stream = torch.cuda.current_stream(X16.device).cuda_stream
+    us_quantize_f16(X16.data_ptr(), X16.stride(0), N, K, amax.data_ptr(), Xq.data_ptr(), sc.data_ptr(), stream)
+    return Xq, sc
+
+
 class SparseWeight:
     """An encoded weight on the current CUDA device. Torch tensors are used only as device memory."""
 
@@ -206,6 +260,21 @@ class SparseWeight:
             stream = torch.cuda.current_stream(X.device).cuda_stream
         us_spmm(self.handle, X.data_ptr(), N, x_scale.data_ptr() if x_scale is not None else None,
                 out.data_ptr(), stream)
+        return out
+
+    def spmm_requant(self, X16, N: int, x_amax, out=None, y_amax=None, amax_range=None, stream=None):
+        """X16: device float16 tensor or view, (N, K) with unit column stride; x_amax: device int32
+        (N,) from absmax_f16 or an earlier call's y_amax. Returns the (N, M) float16 output; if
+        y_amax (device int32 (N,)) is given it receives the absmax of columns amax_range of it."""
+        import torch
+        assert X16.dtype == torch.float16 and X16.stride(1) == 1 and X16.shape[1] == self.K
+        if out is None:
+            out = torch.empty((N, self.M), device=X16.device, dtype=torch.float16)
+        if stream is None:
+            stream = torch.cuda.current_stream(X16.device).cuda_stream
+        m0, m1 = amax_range if amax_range is not None else (0, self.M)
+        us_spmm_requant(self.handle, X16.data_ptr(), X16.stride(0), x_amax.data_ptr(), N, out.data_ptr(),
+                        y_amax.data_ptr() if y_amax is not None else None, m0, m1, stream)
         return out
 
     def check(self):

@@ -10,7 +10,7 @@ PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libunionsparse.so"
 SOURCES = [CSRC / "us_api.cu", CSRC / "us_encode.cpp"]
-HEADERS = [CSRC / "us_host.h", CSRC / "us_spmm_kernel.cuh", PKG.parent / "include" / "unionsparse.h"]
+HEADERS = [CSRC / "us_host.h", CSRC / "us_spmm_kernel.cuh", CSRC / "us_quant_kernels.cuh", PKG.parent / "include" / "unionsparse.h"]
 
 
 def nvcc_command(out: Path, verbose: bool = False) -> list[str]:

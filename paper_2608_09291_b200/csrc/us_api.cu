@@ -9,6 +9,7 @@
 
 #include "us_host.h"
 #include "us_spmm_kernel.cuh"
+#include "us_quant_kernels.cuh"
 
 struct us_handle {
     us::HostMatrix host;
@@ -83,7 +84,7 @@ int segs_per_range(const us::HostMatrix& hm, int nt, int limit, int64_t min_rang
     const int64_t n_segs = hm.n_segs;
     const int slot = (int)((hm.max_item_bytes + 256u + 127u) & ~127u);
     const int acc = nt * 512 * 2 <= kLocalAccBudget ? kLocalAccBudget : 0;
-    const int other = 256 * 8 * 4 + (int)us::kLutScratchBytes + acc + 2 * us::kOffTable * 4 + 1024;
+    const int other = 256 * 8 * 4 + (int)us::kLutScratchBytes + acc + 2 * us::kOffTable * 4 + 1280;
     for (int64_t r = std::max<int64_t>(1, min_ranges); r <= n_segs; ++r) {
         // A single range is worth more (no partial sums leave the CTA when the cuts fall on strip
         // boundaries): it may cost two more warps. Measured on 4096 x 11008, N = 8: one range with
@@ -109,7 +110,7 @@ bool plan_launch(const us_handle* h, int N, LaunchGeom* g)
     int lut_rep = 32;
     auto fixed_for = [&](int rep) {
         return 256 * rep * 4 + (int)us::kLutScratchBytes + (int)x_bytes(g->nt, G, h->host.fmt.K_L, g->xp) + G * g->nt * 8 * 4 +
-                           32 * 4 + s_local * (g->nt * 128 + 1) * 4 + 2 * us::kOffTable * 4 + 128;
+                           us::kClaimWords * 4 + s_local * (g->nt * 128 + 1) * 4 + 2 * us::kOffTable * 4 + 128;
     };
     int fixed_base = fixed_for(lut_rep);
     const int limit = h->max_smem > 0 ? h->max_smem : 227 * 1024;
@@ -185,7 +186,7 @@ void plan_classes(us_handle* h, int n_cta, std::vector<uint32_t> (&sched)[4])
                     if (pass == 0 && need <= kLocalAccBudget) { *s_local = worst; return G; }
                     if (pass == 1 && need <= kLocalAccCap) {
                         const int slot = (int)((h->host.max_item_bytes + 256u + 127u) & ~127u);
-                        const int64_t fixed = 256 * 8 * 4 + (int64_t)us::kLutScratchBytes + need + 2 * us::kOffTable * 4 + 1024 +
+                        const int64_t fixed = 256 * 8 * 4 + (int64_t)us::kLutScratchBytes + need + 2 * us::kOffTable * 4 + 1280 +
                                               x_bytes(nt, G, h->host.fmt.K_L, xp) + (int64_t)G * nt * 32;
                         if ((limit - fixed) / slot >= 11) { *s_local = worst; return G; }
                     }
@@ -338,8 +339,18 @@ us_status check_spmm_args(const us_handle* h, const void* X, int32_t N, const vo
 
 // Fills the kernel parameters and launches: the one code path behind us_spmm and
 // us_spmm_static_scratch (they differ only in where the split-K scratch lives).
+// What a chained call adds to the plain one: fp16 activations quantised while they are staged, and
+// the per-token absmax of a range of output rows left for the next call.
+struct ChainArgs {
+    const void* X16 = nullptr;
+    int64_t ldx = 0;
+    const void* x_amax = nullptr;
+    void* y_amax = nullptr;
+    int64_t m0 = 0, m1 = 0;
+};
+
 us_status enqueue_spmm(us_handle* h, const void* X, int32_t N, const void* x_scale, void* Y, cudaStream_t st,
-                       int32_t* acc, uint32_t* cnt, bool timers)
+                       int32_t* acc, uint32_t* cnt, bool timers, const ChainArgs* chain = nullptr)
 {
     LaunchGeom g;
     if (!plan_launch(h, N, &g)) return US_ERR_UNSUPPORTED;
@@ -373,6 +384,15 @@ us_status enqueue_spmm(us_handle* h, const void* X, int32_t N, const void* x_sca
     p.slot_bytes = g.slot_bytes;
     p.x_fast = (hm.K % 32 == 0) ? 2 : (hm.K % 8 == 0) ? 1 : 0;
     p.fp16_out = x_scale ? 1 : 0;
+    p.X16 = nullptr; p.x_amax = nullptr; p.y_amax = nullptr; p.ldx16 = 0; p.amax_m0 = p.amax_m1 = 0;
+    if (chain) {
+        p.X16 = static_cast<const uint16_t*>(chain->X16);
+        p.x_amax = static_cast<const uint32_t*>(chain->x_amax);
+        p.y_amax = static_cast<uint32_t*>(chain->y_amax);
+        p.ldx16 = chain->ldx;
+        p.amax_m0 = (int32_t)chain->m0; p.amax_m1 = (int32_t)chain->m1;
+        p.fp16_out = 1;
+    }
     p.wait_ns_hi = h->wait_ns_hi;
     p.withhold = h->withhold;
 
@@ -569,6 +589,60 @@ us_status us_spmm_static_scratch(us_handle* h, const void* X, int32_t N, const v
     if (e != cudaSuccess) { h->sticky = e; return US_ERR_CUDA; }
     return enqueue_spmm(h, X, N, x_scale, Y, st, reinterpret_cast<int32_t*>(scratch),
                         reinterpret_cast<uint32_t*>(scratch + acc_bytes), false);
+}
+
+// ---- chained calls: fp16 in, INT4 inside, fp16 out ---------------------------------------------
+us_status us_spmm_requant(us_handle* h, const void* X16, int64_t ldx, const void* x_amax, int32_t N, void* Y16,
+                          void* y_amax, int64_t amax_m0, int64_t amax_m1, void* stream)
+{
+    if (!h || !X16 || !x_amax || !Y16 || N < 1 || N > h->max_N) return US_ERR_INVALID_ARG;
+    if (!h->on_device) return US_ERR_UNSUPPORTED;
+    if (!h->d_w_scale) return US_ERR_INVALID_ARG;   // fp16 output needs the weight scales
+    if (ldx < h->host.K) return US_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(X16) % 2 || reinterpret_cast<uintptr_t>(Y16) % 2 ||
+        reinterpret_cast<uintptr_t>(x_amax) % 4 || reinterpret_cast<uintptr_t>(y_amax) % 4) return US_ERR_INVALID_ARG;
+    if (y_amax && (amax_m0 < 0 || amax_m1 > h->host.M || amax_m0 > amax_m1)) return US_ERR_INVALID_ARG;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return US_ERR_CUDA;
+    if (dev != h->device) return US_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (y_amax) {   // the kernel combines with atomic max: the words start at zero
+        const cudaError_t e = cudaMemsetAsync(y_amax, 0, (size_t)N * sizeof(uint32_t), st);
+        if (e != cudaSuccess) { h->sticky = e; return US_ERR_CUDA; }
+    }
+    ChainArgs c;
+    c.X16 = X16; c.ldx = ldx; c.x_amax = x_amax; c.y_amax = y_amax; c.m0 = amax_m0; c.m1 = amax_m1;
+    return enqueue_spmm(h, X16, N, nullptr, Y16, st, h->d_acc, h->d_cnt, h->timers_on, &c);
+}
+
+us_status us_absmax_f16(const void* X16, int64_t ldx, int32_t N, int64_t K, void* amax, void* stream)
+{
+    if (!X16 || !amax || N < 1 || N > 65535 || K < 1 || ldx < K) return US_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(X16) % 2 || reinterpret_cast<uintptr_t>(amax) % 4) return US_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(amax, 0, (size_t)N * sizeof(uint32_t), st) != cudaSuccess) { cudaGetLastError(); return US_ERR_CUDA; }
+    const int64_t units = (K + 7) / 8;
+    const unsigned gx = (unsigned)std::max<int64_t>(1, std::min<int64_t>(64, (units + 255) / 256));
+    us::us_absmax_f16_kernel<<<dim3(gx, (unsigned)N), 256, 0, st>>>(static_cast<const uint16_t*>(X16), ldx, K,
+                                                                    static_cast<uint32_t*>(amax));
+    if (cudaGetLastError() != cudaSuccess) return US_ERR_CUDA;
+    return US_OK;
+}
+
+us_status us_quantize_f16(const void* X16, int64_t ldx, int32_t N, int64_t K, const void* amax, void* Xq,
+                          void* x_scale, void* stream)
+{
+    if (!X16 || !amax || !Xq || N < 1 || N > 65535 || K < 1 || ldx < K) return US_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(X16) % 2 || reinterpret_cast<uintptr_t>(amax) % 4 ||
+        reinterpret_cast<uintptr_t>(x_scale) % 2) return US_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int64_t units = (K + 7) / 8;
+    const unsigned gx = (unsigned)std::max<int64_t>(1, std::min<int64_t>(64, (units + 255) / 256));
+    us::us_quantize_f16_kernel<<<dim3(gx, (unsigned)N), 256, 0, st>>>(static_cast<const uint16_t*>(X16), ldx, K,
+                                                                      static_cast<const uint32_t*>(amax),
+                                                                      static_cast<uint8_t*>(Xq), static_cast<uint16_t*>(x_scale));
+    if (cudaGetLastError() != cudaSuccess) return US_ERR_CUDA;
+    return US_OK;
 }
 
 us_status us_last_error(us_handle* h)

@@ -38,6 +38,18 @@ def make_x(K: int, N_max: int, seed: int) -> np.ndarray:
     return rng.integers(-8, 8, (N_max, K)).astype(np.int8)
 
 
+def make_x_f16(K: int, N_max: int, seed: int, outliers: bool = True) -> np.ndarray:
+    """fp16 activations for the chained calls, token-major (N_max, K): normal draws with a
+    per-token spread ~U(0.2, 3) and (optionally) a few channels 8x larger, the usual shape of LLM
+    hidden states."""
+    rng = np.random.default_rng([seed, _X_STREAM + 2])
+    x = rng.standard_normal((N_max, K)) * rng.uniform(0.2, 3.0, (N_max, 1))
+    if outliers and K >= 64:
+        ch = rng.choice(K, size=max(1, K // 256), replace=False)
+        x[:, ch] *= 8.0
+    return x.astype(np.float16)
+
+
 def make_scales(M: int, N_max: int, seed: int):
     """fp16 per-output-channel weight scales ~U(0.005,0.02) and per-token activation scales
     ~U(0.01,0.05)."""
@@ -45,6 +57,14 @@ def make_scales(M: int, N_max: int, seed: int):
     s_w = rng.uniform(0.005, 0.02, M).astype(np.float16)
     s_x = rng.uniform(0.01, 0.05, N_max).astype(np.float16)
     return s_w, s_x
+
+
+def make_chain_weight_scales(M: int, K: int, seed: int) -> np.ndarray:
+    """Weight scales for a chain of projections: those of make_scales times 16 / sqrt(K), which
+    keeps the magnitude of the activations about level from one projection to the next (the job
+    the normalisation layers do in a real decoder), so that a chain stays inside the fp16 range."""
+    s_w, _ = make_scales(M, 1, seed)
+    return (s_w.astype(np.float64) * 16.0 / np.sqrt(K)).astype(np.float16)
 
 
 # The synthetic configurations of the build's target (name -> list of cases).

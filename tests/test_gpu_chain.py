@@ -1,0 +1,178 @@
+"""Chained calls (fp16 in, per-token INT4 inside, fp16 out) against the CPU oracle. The quantised
+codes, steps and absmax words are integers decided in fp32 on both sides: they must agree bit for
+bit. The fp16 outputs are checked stage by stage from the device's own previous output, within
+max(2e-3 relative, 1 fp16 ulp) of the exactly rounded reference."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2608_09291_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+@pytest.fixture(scope="module")
+def b():
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    from paper_2608_09291_b200 import binding
+    torch.cuda.set_device(0)
+    return binding
+
+
+def _unpack(Xq: np.ndarray, K: int) -> np.ndarray:
+    nib = np.empty((Xq.shape[0], 2 * Xq.shape[1]), dtype=np.int16)
+    nib[:, 0::2] = Xq & 0xF
+    nib[:, 1::2] = Xq >> 4
+    nib = nib[:, :K]
+    return np.where(nib >= 8, nib - 16, nib).astype(np.int8)
+
+
+def _amax_words(a16: np.ndarray) -> np.ndarray:
+    return a16.view(np.uint16).astype(np.int32)
+
+
+@pytest.mark.parametrize("N,K,pad,off", [(8, 4096, 0, 0), (16, 5120, 10240, 5120), (5, 1000, 24, 0),
+                                         (3, 1001, 6, 1), (1, 7, 0, 0), (64, 256, 0, 0)])
+def test_absmax_and_quantize_bit_exact(b, N, K, pad, off):
+    """Aligned and unaligned rows, ragged K, a column window of a wider buffer."""
+    full = workloads.make_x_f16(K + pad, N, seed=900 + K)
+    full[0, off] = 0.0
+    if N > 2:
+        full[2, off:off + K] = 0.0                       # an all-zero token
+        full[1, off:off + K] *= np.float16(2.0 ** -14)   # a token deep in the small range
+    Xd = torch.from_numpy(full).cuda()
+    view = Xd[:, off:off + K]
+    x = full[:, off:off + K]
+    amax = b.absmax_f16(view)
+    Xq, sc = b.quantize_f16(view, amax)
+    torch.cuda.synchronize()
+    a_ref = oracle.absmax_f16(x)
+    assert np.array_equal(amax.cpu().numpy(), _amax_words(a_ref))
+    q_ref, s_ref = oracle.requant_int4(x)
+    assert np.array_equal(sc.cpu().numpy().view(np.uint16), s_ref.view(np.uint16))
+    assert np.array_equal(_unpack(Xq.cpu().numpy(), K), q_ref)
+
+
+def _check_requant_call(b, sw, W, s_w, x16, N, m0, m1, reps=2):
+    """One chained call on activations x16 (numpy (N, K) fp16): output within the bar, absmax words
+    exact for the values the device stored."""
+    Xd = torch.from_numpy(np.ascontiguousarray(x16)).cuda()
+    amax = b.absmax_f16(Xd)
+    y_amax = torch.full((N,), -1, dtype=torch.int32, device="cuda")
+    q, s = oracle.requant_int4(x16)
+    ref = oracle.spmm_dense(W, q)
+    for rep in range(reps):
+        Y = sw.spmm_requant(Xd, N, amax, y_amax=y_amax, amax_range=(m0, m1))
+        torch.cuda.synchronize()
+        sw.check()
+        got = Y.cpu().numpy()
+        ok = oracle.fp16_within_tolerance(got, ref, s_w, s, rel=2e-3)
+        assert ok.all(), f"rep {rep}: {int((~ok).sum())} fp16 outputs outside tolerance"
+        assert np.array_equal(y_amax.cpu().numpy(), _amax_words(oracle.absmax_f16(got, m0, m1))), f"rep {rep}"
+    return got
+
+
+@pytest.mark.parametrize("M,K,N,s,rng_m", [
+    (1024, 1024, 8, 0.5, (0, 1024)),
+    (4096, 4096, 1, 0.5, (100, 3000)),
+    (4096, 4096, 16, 0.3, (0, 4096)),
+    (2000, 1000, 5, 0.5, (7, 1993)),        # ragged rows and columns
+    (1030, 2056, 12, 0.6, (0, 0)),          # empty range: the words stay zero
+    (5120, 13824, 16, 0.5, (0, 5120)),      # the 13B down projection
+    (11008, 4096, 32, 0.5, (11008 - 16, 11008)),
+    (4096, 11008, 32, 0.5, (0, 4096)),      # global split-K path
+    (4096, 4096, 64, 0.5, (1, 4095)),
+])
+def test_spmm_requant(b, M, K, N, s, rng_m):
+    seed = 700 + M % 97 + K % 89 + N
+    W = workloads.make_weight(M, K, s, seed=seed)
+    s_w, _ = workloads.make_scales(M, N, seed=seed)
+    x16 = workloads.make_x_f16(K, N, seed=seed)
+    sw = b.SparseWeight(W, s_w, max_N=N)
+    try:
+        _check_requant_call(b, sw, W, s_w, x16, N, *rng_m)
+        # the plain entry point fed with the separately quantised codes gives the same fp16 values
+        Xd = torch.from_numpy(x16).cuda()
+        amax = b.absmax_f16(Xd)
+        Xq, sc = b.quantize_f16(Xd, amax)
+        y_plain = sw.spmm(Xq, N, sc)
+        y_chain = sw.spmm_requant(Xd, N, amax)
+        torch.cuda.synchronize()
+        sw.check()
+        assert torch.equal(y_plain, y_chain)
+    finally:
+        sw.close()
+
+
+def test_requant_argument_errors(b):
+    W = workloads.make_weight(256, 256, 0.5, seed=5)
+    s_w, _ = workloads.make_scales(256, 8, seed=5)
+    sw = b.SparseWeight(W, s_w, max_N=8)
+    bare = b.SparseWeight(W, None, max_N=8)
+    try:
+        X = torch.zeros((8, 256), dtype=torch.float16, device="cuda")
+        a = torch.zeros(8, dtype=torch.int32, device="cuda")
+        Y = torch.zeros((8, 256), dtype=torch.float16, device="cuda")
+        call = b._lib.us_spmm_requant
+        assert call(sw.handle, X.data_ptr(), 255, a.data_ptr(), 8, Y.data_ptr(), None, 0, 0, None) == 1   # ldx < K
+        assert call(sw.handle, X.data_ptr(), 256, a.data_ptr(), 9, Y.data_ptr(), None, 0, 0, None) == 1   # N > max_N
+        assert call(sw.handle, X.data_ptr(), 256, a.data_ptr(), 8, Y.data_ptr(), a.data_ptr(), 0, 257, None) == 1
+        assert call(sw.handle, X.data_ptr(), 256, a.data_ptr(), 8, Y.data_ptr(), a.data_ptr(), 9, 3, None) == 1
+        assert call(sw.handle, None, 256, a.data_ptr(), 8, Y.data_ptr(), None, 0, 0, None) == 1
+        assert call(bare.handle, X.data_ptr(), 256, a.data_ptr(), 8, Y.data_ptr(), None, 0, 0, None) == 1  # no weight scales
+        assert b._lib.us_absmax_f16(X.data_ptr(), 100, 8, 256, a.data_ptr(), None) == 1
+        assert b._lib.us_quantize_f16(X.data_ptr(), 256, 0, 256, a.data_ptr(), Y.data_ptr(), None, None) == 1
+        torch.cuda.synchronize()
+        sw.check()
+    finally:
+        sw.close()
+        bare.close()
+
+
+@pytest.mark.parametrize("j,s", [(0, 0.3), (1, 0.5), (2, 0.7)])
+def test_layer_13b_chain(b, j, s):
+    """The projections of one 13B-shaped decoder layer as a chain of four launches on one stream,
+    no synchronisation in between: [Q;K;V] stacked (15360 x 5120) -> O (5120 x 5120, reads the Q
+    columns) -> [gate;up] stacked (27648 x 5120) -> down (5120 x 13824, reads the gate columns).
+    The attention and the gating between them are not this library's work: the chain carries the
+    data flow and the re-quantisation. Each stage is checked against the oracle from the device's
+    own previous output."""
+    N, H, F = 16, 5120, 13824
+    shapes = [("qkv", 3 * H, H, (0, H)), ("o", H, H, (0, H)), ("gate_up", 2 * F, H, (0, F)), ("down", H, F, (0, 0))]
+    mats = []
+    try:
+        for i, (name, M, K, rng_m) in enumerate(shapes):
+            seed = 800 + 10 * j + i
+            W = workloads.make_weight(M, K, s, seed=seed)
+            s_w = workloads.make_chain_weight_scales(M, K, seed=seed)
+            mats.append(dict(W=W, s_w=s_w, sw=b.SparseWeight(W, s_w, max_N=N), M=M, K=K, rng=rng_m,
+                             Y=torch.zeros((N, M), dtype=torch.float16, device="cuda"),
+                             amax=torch.zeros(N, dtype=torch.int32, device="cuda")))
+        x0 = workloads.make_x_f16(H, N, seed=800 + 10 * j)
+        X0 = torch.from_numpy(x0).cuda()
+        a0 = torch.zeros(N, dtype=torch.int32, device="cuda")
+        for rnd in range(2):
+            b.absmax_f16(X0, out=a0)
+            src, src_amax = X0, a0
+            for m in mats:
+                m["sw"].spmm_requant(src, N, src_amax, out=m["Y"], y_amax=m["amax"], amax_range=m["rng"])
+                src, src_amax = m["Y"][:, m["rng"][0]:m["rng"][1]], m["amax"]
+            torch.cuda.synchronize()
+            prev = x0
+            for m in mats:
+                m["sw"].check()
+                got = m["Y"].cpu().numpy()
+                q, st = oracle.requant_int4(prev)
+                ref = oracle.spmm_dense(m["W"], q)
+                assert np.isfinite(got).all() and np.abs(got).max() > 0
+                ok = oracle.fp16_within_tolerance(got, ref, m["s_w"], st, rel=2e-3)
+                assert ok.all(), f"round {rnd}: {int((~ok).sum())} outputs outside tolerance"
+                m0, m1 = m["rng"]
+                assert np.array_equal(m["amax"].cpu().numpy(), _amax_words(oracle.absmax_f16(got, m0, m1)))
+                prev = got[:, m0:m1]
+    finally:
+        for m in mats:
+            m["sw"].close()
