@@ -532,6 +532,7 @@ def sweep(binding, torch, workloads, l2, peak_gbs):
     run_case("ffn70b_up_paired", 28672, 8192, 0.6, 500, [8], [False], flags=binding.US_ENCODE_PAIR_ROWS)
     for s in (0.3, 0.5, 0.7):                                                                  # config 4
         rows.append(layer_chain(binding, torch, workloads, l2, s))
+        rows.append(layer_chain_requant(binding, torch, workloads, l2, s))
     return rows
 
 
@@ -592,6 +593,76 @@ def layer_chain(binding, torch, workloads, l2, sparsity=0.5):
            "pct_of_8tbs": 100 * alg / t / 1e9 / CONTRACT_PEAK_GBS, "frac_of_measured": alg / t / 1e9 / measured_peaks()[0],
            "dense_equiv_tops": 2.0 * sum(m * k for m, k in shapes) * N / t / 1e12, "replicas": len(copies),
            "pmr": copies[0][0].stats["pmr"], "launches_per_unit": len(shapes)}
+    for layer in copies:
+        for sw in layer:
+            sw.close()
+    torch.cuda.empty_cache()
+    return row
+
+
+def layer_chain_requant(binding, torch, workloads, l2, sparsity=0.5):
+    """The same seven weight matrices as layer_chain, as a chain of four chained calls: [Q;K;V]
+    stacked into one 15360 x 5120 matrix, O, [gate;up] stacked into 27648 x 5120, down. Activations
+    travel as fp16; each call quantises its input per token to INT4 while staging it and leaves the
+    absmax its successor needs (O reads the Q columns, down reads the gate columns: the attention
+    and the gating in between are not this library's work). One CUDA graph, several layer copies."""
+    H, F, N = 5120, 13824, 16
+    base = [(H, H)] * 4 + [(F, H)] * 2 + [(H, F)]
+    Ws = [workloads.make_weight(m, k, sparsity, 410 + i) for i, (m, k) in enumerate(base)]
+    groups = [([0, 1, 2], (0, H)), ([3], (0, H)), ([4, 5], (0, F)), ([6], (0, 0))]
+    mats = []
+    for g, (idx, rng) in enumerate(groups):
+        W = np.concatenate([Ws[i] for i in idx], axis=0)
+        mats.append((W, workloads.make_chain_weight_scales(W.shape[0], W.shape[1], 410 + g), rng))
+    del Ws
+    layer_bytes, copies = 0, []
+    while layer_bytes * len(copies) < 3.2 * l2 or len(copies) < 2:
+        layer = [binding.SparseWeight(W, s_w, max_N=N) for W, s_w, _ in mats]
+        layer_bytes = sum(sw.stats["bytes_total"] for sw in layer)
+        copies.append(layer)
+    alg = sum(sw.stats["bytes_payload"] + sw.stats["bytes_bitmap"] + sw.stats["bytes_offsets"] + 2 * sw.M +
+              2 * N * sw.K + 2 * N * sw.M + 8 * N for sw in copies[0])
+    X0 = torch.from_numpy(workloads.make_x_f16(H, N, 77)).cuda()
+    a0 = binding.absmax_f16(X0)
+    outs = [torch.empty((N, W.shape[0]), dtype=torch.float16, device="cuda") for W, _, _ in mats]
+    amaxs = [torch.zeros(N, dtype=torch.int32, device="cuda") for _ in mats]
+
+    def enqueue():
+        for layer in copies:
+            src, src_amax = X0, a0
+            for sw, (_, _, rng), Y, am in zip(layer, mats, outs, amaxs):
+                sw.spmm_requant(src, N, src_amax, out=Y, y_amax=am, amax_range=rng)
+                src, src_amax = Y[:, rng[0]:rng[1]], am
+
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        enqueue()
+    torch.cuda.current_stream().wait_stream(s)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        enqueue()
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 20
+    e0.record()
+    for _ in range(reps):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    for layer in copies:
+        for sw in layer:
+            sw.check()
+    assert bool(torch.isfinite(outs[-1]).all())
+    t = e0.elapsed_time(e1) * 1e-3 / (reps * len(copies))
+    row = {"case": "layer13b_chain_requant", "M": 0, "K": 0, "sparsity": sparsity, "N": N, "out": "fp16", "us": t * 1e6,
+           "alg_bytes": alg, "stored_bytes": layer_bytes, "gbs": alg / t / 1e9,
+           "pct_of_8tbs": 100 * alg / t / 1e9 / CONTRACT_PEAK_GBS, "frac_of_measured": alg / t / 1e9 / measured_peaks()[0],
+           "dense_equiv_tops": 2.0 * sum(m * k for m, k in base) * N / t / 1e12, "replicas": len(copies),
+           "pmr": copies[0][0].stats["pmr"], "launches_per_unit": len(mats)}
     for layer in copies:
         for sw in layer:
             sw.close()
@@ -683,6 +754,18 @@ def torchrun_command(argv, gpus: int, port: int = 29541):
             "--master-addr", "127.0.0.1", "--master-port", str(port), str(Path(__file__).resolve())] + list(argv)
 
 
+def run_chain():
+    import torch
+    from paper_2608_09291_b200 import build as libbuild
+    libbuild.build()
+    from paper_2608_09291_b200 import binding, workloads
+    torch.cuda.set_device(0)
+    l2 = torch.cuda.get_device_properties(0).L2_cache_size or L2_BYTES_FALLBACK
+    for s in (0.3, 0.5, 0.7):
+        print(json.dumps(layer_chain(binding, torch, workloads, l2, s)))
+        print(json.dumps(layer_chain_requant(binding, torch, workloads, l2, s)))
+
+
 def main(argv=None):
     argv = list(sys.argv[1:] if argv is None else argv)
     ap = argparse.ArgumentParser()
@@ -693,6 +776,8 @@ def main(argv=None):
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--only", default=None, metavar="M,K,s,N[,int32|fp16[,K_L[,N_max]]]",
                     help="time one case only, with the kernel's stage timers: the small run of the ncu captures")
+    ap.add_argument("--chain", action="store_true",
+                    help="time only the 13B-shaped layer, as seven plain calls and as a chain of four chained calls")
     args = ap.parse_args(argv)
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -711,6 +796,9 @@ def main(argv=None):
         return
     if args.only:
         run_only(args)
+        return
+    if args.chain:
+        run_chain()
         return
     run_ours(args, rank, local_rank, world)
 

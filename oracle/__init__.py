@@ -16,10 +16,12 @@ What each function follows:
   absmax_f16           max |y| per token over a column range, exact in fp16
   requant_int4         per-token symmetric INT4 re-quantisation of an fp16 activation. The paper
                        takes INT4 activations as given (W4A4, Sec. VII-A) and defines no
-                       quantiser; the reading used here is the plain symmetric absmax one:
-                       s = max(RN_fp16(fp32(amax) / 7), 2^-24), code = clamp(RNE(fp32(y) /
-                       fp32(s)), -8, 7), division and rounding in fp32 (the kernel's precision:
-                       floating point decides an integer here, so both sides fix it)
+                       quantiser; the reading used here is the plain symmetric absmax one with
+                       a reciprocal step: s = RN_fp16(fp32(amax) / 7) is the dequantisation
+                       scale, inv = min(RN_fp16(7 / fp32(amax)), 65504) (65504 when amax = 0),
+                       code = clamp(RNE(y * inv), -8, 7) with the product of the two fp16
+                       numbers taken exactly (it fits fp32). Floating point decides an integer
+                       here, so this precision is part of the definition on both sides.
 """
 from __future__ import annotations
 
@@ -195,14 +197,22 @@ def absmax_f16(y16: np.ndarray, m0: int = 0, m1: int | None = None) -> np.ndarra
     return np.abs(y).max(axis=1).astype(np.float16)
 
 
-FP16_TINY = np.float16(2.0 ** -24)   # the smallest positive fp16
+FP16_MAX = np.float16(65504.0)
 
 
 def requant_scale(amax16: np.ndarray) -> np.ndarray:
-    """s[n] = max(RN_fp16(fp32(amax[n]) / fp32(7)), 2^-24): the quantisation step per token."""
+    """s[n] = RN_fp16(fp32(amax[n]) / fp32(7)): the dequantisation scale per token."""
     a = np.asarray(amax16, dtype=np.float16).astype(np.float32)
-    s = (a / np.float32(7.0)).astype(np.float16)
-    return np.maximum(s, FP16_TINY)
+    return (a / np.float32(7.0)).astype(np.float16)
+
+
+def requant_inverse(amax16: np.ndarray) -> np.ndarray:
+    """inv[n] = min(RN_fp16(fp32(7) / fp32(amax[n])), 65504); 65504 for amax = 0."""
+    a = np.asarray(amax16, dtype=np.float16).astype(np.float32)
+    with np.errstate(divide="ignore", over="ignore"):
+        inv = np.float32(7.0) / a                       # +inf for amax = 0
+        inv16 = inv.astype(np.float16)                  # overflows to +inf above 65504 (+ half an ulp)
+    return np.minimum(inv16, FP16_MAX)
 
 
 def requant_int4(y16: np.ndarray, amax16: np.ndarray | None = None):
@@ -211,10 +221,10 @@ def requant_int4(y16: np.ndarray, amax16: np.ndarray | None = None):
     y = np.asarray(y16, dtype=np.float16)
     if amax16 is None:
         amax16 = absmax_f16(y)
-    s = requant_scale(amax16)
-    r = y.astype(np.float32) / s.astype(np.float32)[:, None]       # IEEE fp32 division
+    inv = requant_inverse(amax16)
+    r = y.astype(np.float32) * inv.astype(np.float32)[:, None]     # exact: 11-bit x 11-bit significands
     q = np.clip(np.rint(r), -8, 7).astype(np.int8)                  # rint: ties to even
-    return q, s
+    return q, requant_scale(amax16)
 
 
 def num_threads() -> int:

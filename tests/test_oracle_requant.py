@@ -20,21 +20,22 @@ def _cases():
         key, rest = line.split(None, 1)
         cur[key] = rest.split()
         if key == "q":
-            yield (np.array([float(v) for v in cur["y"]], dtype=np.float64),
-                   int(cur["s"][0], 16), np.array([int(v) for v in cur["q"]], dtype=np.int8))
+            yield (np.array([float(v) for v in cur["y"]], dtype=np.float64), int(cur["s"][0], 16),
+                   int(cur["inv"][0], 16), np.array([int(v) for v in cur["q"]], dtype=np.int8))
             cur = {}
 
 
 def test_hand_worked_cases():
     n = 0
-    for y, s_bits, q_exp in _cases():
+    for y, s_bits, inv_bits, q_exp in _cases():
         y16 = y.astype(np.float16)
         assert np.array_equal(y16.astype(np.float64), y), "fixture value not exact in fp16"
         q, s = oracle.requant_int4(y16[None, :])
         assert int(s.view(np.uint16)[0]) == s_bits
+        assert int(oracle.requant_inverse(oracle.absmax_f16(y16[None, :])).view(np.uint16)[0]) == inv_bits
         assert np.array_equal(q[0], q_exp)
         n += 1
-    assert n == 5
+    assert n == 6
 
 
 def _round_half_even(fr: Fraction) -> int:
@@ -61,19 +62,21 @@ def _fp16_nearest(fr: Fraction) -> np.float16:
 
 @pytest.mark.parametrize("seed", [0, 1, 2])
 def test_against_exact_rational_arithmetic(seed):
-    """fp16 operands have 11-bit significands, so a quotient that is not a tie stays farther from
-    the tie than fp32 rounding can move it: the fp32 decision must equal the exact one."""
+    """Scale and reciprocal are the correctly rounded fp16 quotients, and every code is the
+    round-half-even of the exact rational product y * inv."""
     rng = np.random.default_rng(seed)
     scale = [1.0, 37.5, 2.0 ** -9][seed]
     y16 = (rng.standard_normal((6, 97)) * scale).astype(np.float16)
     y16[0, :8] = np.float16(scale) * np.array([0.5, 1.5, 2.5, 3.5, -0.5, -1.5, -2.5, 7], np.float16)
     q, s = oracle.requant_int4(y16)
+    inv = oracle.requant_inverse(oracle.absmax_f16(y16))
     for n in range(y16.shape[0]):
         amax = max(abs(Fraction(float(v))) for v in y16[n])
-        s_exact = max(_fp16_nearest(amax / 7), oracle.FP16_TINY) if amax else oracle.FP16_TINY
-        assert s[n] == s_exact
+        assert s[n] == _fp16_nearest(amax / 7)
+        inv_exact = _fp16_nearest(Fraction(7) / amax)
+        assert np.isfinite(inv_exact) and inv[n] == inv_exact
         for m in range(y16.shape[1]):
-            r = _round_half_even(Fraction(float(y16[n, m])) / Fraction(float(s_exact)))
+            r = _round_half_even(Fraction(float(y16[n, m])) * Fraction(float(inv_exact)))
             assert q[n, m] == min(7, max(-8, r)), (n, m)
 
 
@@ -85,8 +88,8 @@ def test_invariants():
     # the extreme element lands on +-7, nothing reaches -8 in the normal range
     idx = np.abs(y16.astype(np.float64)).argmax(axis=1)
     assert np.all(np.abs(q[np.arange(16), idx]) == 7) and q.min() >= -7 and q.max() <= 7
-    # reconstruction error at most half a step
-    assert np.all(np.abs(q * sf - y16.astype(np.float64)) <= 0.5 * sf * (1 + 1e-6))
+    # reconstruction error at most half a step (s * inv = 1 within two fp16 roundings)
+    assert np.all(np.abs(q * sf - y16.astype(np.float64)) <= 0.5 * sf * (1 + 32 * 2.0 ** -11))
     # odd symmetry, and exact covariance under a power-of-two scaling
     qn, sn = oracle.requant_int4(-y16)
     assert np.array_equal(qn, -q) and np.array_equal(sn, s)
