@@ -625,7 +625,7 @@ def layer_chain_requant(binding, torch, workloads, l2, sparsity=0.5):
     X0 = torch.from_numpy(workloads.make_x_f16(H, N, 77)).cuda()
     a0 = binding.absmax_f16(X0)
     outs = [torch.empty((N, W.shape[0]), dtype=torch.float16, device="cuda") for W, _, _ in mats]
-    amaxs = [torch.zeros(N, dtype=torch.int32, device="cuda") for _ in mats]
+    amaxs = [binding.new_amax() for _ in mats]
 
     def enqueue():
         for layer in copies:

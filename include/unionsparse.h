@@ -172,30 +172,38 @@ us_status us_last_error(us_handle* h);
  * Chained calls: fp16 activations in, INT4 inside, fp16 out.
  *
  * The paper evaluates the W4A4 kernel on INT4 activations that are given (Sec. VII-A) and defines
- * no activation quantiser; these three calls have no counterpart in it. They let the output of one
- * projection feed the next without a pass over the activations in between. The quantiser is the
- * plain per-token symmetric one:
- *     step[n] = max(RN_fp16(amax[n] / 7), 2^-24),  code = clamp(RNE(x / step[n]), -8, 7),
- * amax[n] = max |x[n][k]| over the quantised columns, the quotients taken in IEEE fp32 (so the codes
- * are reproducible bit for bit), and step[n] is the activation scale of the dequantisation.
+ * no activation quantiser; these three calls have no counterpart in it. They let the fp16 output of
+ * one projection feed the next: the producing kernel's epilogue leaves the per-token absmax, and one
+ * small kernel between the two turns the activations into INT4 codes. The quantiser is the
+ * plain per-token symmetric one with a reciprocal step:
+ *     amax[n]  = max |x[n][k]| over the quantised columns
+ *     scale[n] = RN_fp16(amax[n] / 7)                     (what the dequantisation multiplies by)
+ *     inv[n]   = min(RN_fp16(7 / amax[n]), 65504)         (65504 for amax = 0)
+ *     code     = clamp(RNE(x * inv[n]), -8, 7)            (the fp16 x fp16 product taken exactly)
+ * so the codes are reproducible bit for bit. Tokens with amax below 7 / 65504 lose resolution.
  *
- * us_spmm_requant: Y16[n][m] = RN_fp16(sum_k W[m][k] * code(X16[n][k]) * w_scale[m] * step[n]).
+ * Absmax buffer: US_AMAX_BYTES bytes of device memory, 4-byte aligned, written by us_absmax_f16 or
+ * by a us_spmm_requant (y_amax) and read by the next us_spmm_requant (x_amax). Layout: word 0 = P,
+ * the number of parts; word 64 + 64 * p + n = the fp16 bit pattern of a partial absmax of token n
+ * (p < P, n < 64); amax[n] is the largest of the P words. Writers store every part, so a buffer
+ * never needs clearing. It holds one tensor's absmax at a time.
+ *
+ * us_spmm_requant: Y16[n][m] = RN_fp16(sum_k W[m][k] * code(X16[n][k]) * w_scale[m] * scale[n]).
  *   X16     device, N rows of fp16, row n at X16 + n * ldx (elements), ldx >= K; finite values.
  *           16-byte aligned rows (pointer and ldx % 8 == 0) take the vector path.
- *   x_amax  device, N 32-bit words: the fp16 bit pattern of amax[n] (what us_absmax_f16 or an earlier
- *           us_spmm_requant wrote).
+ *   x_amax  device absmax buffer of X16's quantised columns.
  *   Y16     device, N x M fp16 row-major. The handle must hold weight scales.
- *   y_amax  device, N 32-bit words or NULL. If given, the call sets word n to the fp16 bit pattern of
- *           max |Y16[n][m]| over amax_m0 <= m < amax_m1 (0 for an empty range): the x_amax of a next
- *           call that reads columns [amax_m0, amax_m1) of Y16. It is cleared on the stream before the
- *           kernel starts and must not be the x_amax of this same call.
+ *   y_amax  device absmax buffer or NULL. If given, the call fills it with the absmax of
+ *           Y16[n][m] over amax_m0 <= m < amax_m1 (0 for an empty range): the x_amax of a next
+ *           call that reads columns [amax_m0, amax_m1) of Y16. Must differ from x_amax.
  * Everything else (stream order, workspace, errors, limits on N) is as for us_spmm.
  *
- * us_absmax_f16: amax[n] = max_k |X16[n][k]| for the head of a chain. N <= 65535.
+ * us_absmax_f16: fills an absmax buffer from X16 (N <= 64 tokens, K columns) for the head of a chain.
  * us_quantize_f16: the codes themselves, packed as us_spmm expects X (N x ceil(K/2) bytes, even k in
- *   the low nibble), and the steps as fp16 bit patterns in x_scale (N entries, may be NULL).
+ *   the low nibble), and the scales as fp16 bit patterns in x_scale (N entries, may be NULL).
  * Both take device pointers, run on `stream`, keep no state and allocate nothing.
  */
+#define US_AMAX_BYTES (4 * 64 * (1 + 192))
 us_status us_spmm_requant(us_handle* h, const void* X16, int64_t ldx, const void* x_amax, int32_t N,
                           void* Y16, void* y_amax, int64_t amax_m0, int64_t amax_m1, void* stream);
 us_status us_absmax_f16(const void* X16, int64_t ldx, int32_t N, int64_t K, void* amax, void* stream);

@@ -147,7 +147,7 @@ def us_spmm_requant(h: int, X16_ptr: int, ldx: int, x_amax_ptr: int, N: int, Y16
 
 
 def us_absmax_f16(X16_ptr: int, ldx: int, N: int, K: int, amax_ptr: int, stream: int | None = None):
-    """amax[n] (32-bit words holding fp16 bit patterns) = max_k |X16[n][k]|."""
+    """Fills the absmax buffer at amax_ptr with max_k |X16[n][k]| per token."""
     _check(_lib.us_absmax_f16(X16_ptr, int(ldx), int(N), int(K), amax_ptr, stream), "us_absmax_f16")
 
 
@@ -212,14 +212,30 @@ def pack_int4(X: np.ndarray) -> np.ndarray:
     return np.ascontiguousarray(u[:, 0::2] | (u[:, 1::2] << 4))
 
 
+US_AMAX_BYTES = 4 * 64 * (1 + 192)
+
+
+def new_amax(device="cuda"):
+    """An absmax buffer (device int32 tensor) for the chained calls."""
+    import torch
+    return torch.zeros(US_AMAX_BYTES // 4, device=device, dtype=torch.int32)
+
+
+def amax_values(buf, N: int):
+    """The per-token absmax an absmax buffer holds, as a host uint16 array of fp16 bit patterns."""
+    w = buf.cpu().numpy()
+    parts = int(w[0])
+    return w[64:64 + 64 * parts].reshape(parts, 64)[:, :N].max(axis=0).astype(np.uint16)
+
+
 def absmax_f16(X16, out=None, stream=None):
     """Per-token absmax of a device float16 (N, K) tensor or view (unit column stride), as the
-    int32 words the chained call takes."""
+    absmax buffer the chained call takes."""
     import torch
     assert X16.dtype == torch.float16 and X16.stride(1) == 1
     N, K = X16.shape
     if out is None:
-        out = torch.empty(N, device=X16.device, dtype=torch.int32)
+        out = new_amax(X16.device)
     if stream is None:
         stream = torch.cuda.current_stream(X16.device).cuda_stream
     us_absmax_f16(X16.data_ptr(), X16.stride(0), N, K, out.data_ptr(), stream)
@@ -263,9 +279,9 @@ class SparseWeight:
         return out
 
     def spmm_requant(self, X16, N: int, x_amax, out=None, y_amax=None, amax_range=None, stream=None):
-        """X16: device float16 tensor or view, (N, K) with unit column stride; x_amax: device int32
-        (N,) from absmax_f16 or an earlier call's y_amax. Returns the (N, M) float16 output; if
-        y_amax (device int32 (N,)) is given it receives the absmax of columns amax_range of it."""
+        """X16: device float16 tensor or view, (N, K) with unit column stride; x_amax: absmax buffer
+        from absmax_f16 or an earlier call's y_amax. Returns the (N, M) float16 output; if y_amax
+        (an absmax buffer) is given it receives the absmax of columns amax_range of the output."""
         import torch
         assert X16.dtype == torch.float16 and X16.stride(1) == 1 and X16.shape[1] == self.K
         if out is None:

@@ -31,6 +31,8 @@ struct us_handle {
     int32_t* d_acc = nullptr;
     uint32_t* d_cnt = nullptr;
     uint32_t* d_err = nullptr;
+    uint8_t* d_xq = nullptr;          // chained calls: packed INT4 codes of the activations, then their scales
+    size_t xq_bytes = 0;              // bytes of the codes (the fp16 scales follow, 256-byte aligned)
     unsigned long long* d_timers = nullptr;
     bool timers_on = false;
     size_t acc_bytes = 0, cnt_bytes = 0;
@@ -312,7 +314,7 @@ void free_device(us_handle* h)
 {
     cudaFree(h->d_blob); cudaFree(h->d_item_off);
     cudaFree(h->d_row_order); cudaFree(h->d_w_scale); cudaFree(h->d_acc);
-    cudaFree(h->d_cnt); cudaFree(h->d_err); cudaFree(h->d_timers);
+    cudaFree(h->d_cnt); cudaFree(h->d_err); cudaFree(h->d_timers); cudaFree(h->d_xq);
 }
 
 template <class T>
@@ -339,12 +341,9 @@ us_status check_spmm_args(const us_handle* h, const void* X, int32_t N, const vo
 
 // Fills the kernel parameters and launches: the one code path behind us_spmm and
 // us_spmm_static_scratch (they differ only in where the split-K scratch lives).
-// What a chained call adds to the plain one: fp16 activations quantised while they are staged, and
-// the per-token absmax of a range of output rows left for the next call.
+// What a chained call adds to the plain one: the per-token absmax of a range of output rows, left
+// for the quantiser of the next call.
 struct ChainArgs {
-    const void* X16 = nullptr;
-    int64_t ldx = 0;
-    const void* x_amax = nullptr;
     void* y_amax = nullptr;
     int64_t m0 = 0, m1 = 0;
 };
@@ -384,14 +383,10 @@ us_status enqueue_spmm(us_handle* h, const void* X, int32_t N, const void* x_sca
     p.slot_bytes = g.slot_bytes;
     p.x_fast = (hm.K % 32 == 0) ? 2 : (hm.K % 8 == 0) ? 1 : 0;
     p.fp16_out = x_scale ? 1 : 0;
-    p.X16 = nullptr; p.x_amax = nullptr; p.y_amax = nullptr; p.ldx16 = 0; p.amax_m0 = p.amax_m1 = 0;
+    p.y_amax = nullptr; p.amax_m0 = p.amax_m1 = 0;
     if (chain) {
-        p.X16 = static_cast<const uint16_t*>(chain->X16);
-        p.x_amax = static_cast<const uint32_t*>(chain->x_amax);
         p.y_amax = static_cast<uint32_t*>(chain->y_amax);
-        p.ldx16 = chain->ldx;
         p.amax_m0 = (int32_t)chain->m0; p.amax_m1 = (int32_t)chain->m1;
-        p.fp16_out = 1;
     }
     p.wait_ns_hi = h->wait_ns_hi;
     p.withhold = h->withhold;
@@ -486,6 +481,10 @@ us_status us_encode(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_sca
     if (e == cudaSuccess) e = cudaMemset(h->d_acc, 0, h->acc_bytes);
     if (e == cudaSuccess) e = cudaMalloc((void**)&h->d_cnt, h->cnt_bytes);
     if (e == cudaSuccess) e = cudaMemset(h->d_cnt, 0, h->cnt_bytes);
+    if (e == cudaSuccess && !hm.w_scale.empty()) {   // chained calls need fp16 output, hence weight scales
+        h->xq_bytes = (((size_t)max_N * (size_t)((hm.K + 1) / 2)) + 255) & ~(size_t)255;
+        e = cudaMalloc((void**)&h->d_xq, h->xq_bytes + 256);
+    }
     if (e == cudaSuccess) e = cudaMalloc((void**)&h->d_err, 16);
     if (e == cudaSuccess) e = cudaMemset(h->d_err, 0, 16);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
@@ -592,6 +591,24 @@ us_status us_spmm_static_scratch(us_handle* h, const void* X, int32_t N, const v
 }
 
 // ---- chained calls: fp16 in, INT4 inside, fp16 out ---------------------------------------------
+namespace {
+cudaError_t launch_quantize(const uint16_t* X16, int64_t ldx, int32_t N, int64_t K, const uint32_t* amax, uint8_t* Xq,
+                            uint16_t* x_scale, cudaStream_t st)
+{
+    const int64_t units = (K + 7) / 8;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)std::max<int64_t>(1, std::min<int64_t>(64, (units + 255) / 256)), (unsigned)N);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = pdl_knob() ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, us::us_quantize_f16_kernel, X16, ldx, K, amax, Xq, x_scale);
+}
+}  // namespace
+
 us_status us_spmm_requant(us_handle* h, const void* X16, int64_t ldx, const void* x_amax, int32_t N, void* Y16,
                           void* y_amax, int64_t amax_m0, int64_t amax_m1, void* stream)
 {
@@ -606,24 +623,28 @@ us_status us_spmm_requant(us_handle* h, const void* X16, int64_t ldx, const void
     if (cudaGetDevice(&dev) != cudaSuccess) return US_ERR_CUDA;
     if (dev != h->device) return US_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (y_amax) {   // the kernel combines with atomic max: the words start at zero
-        const cudaError_t e = cudaMemsetAsync(y_amax, 0, (size_t)N * sizeof(uint32_t), st);
-        if (e != cudaSuccess) { h->sticky = e; return US_ERR_CUDA; }
-    }
+    if (y_amax == x_amax) return US_ERR_INVALID_ARG;
     ChainArgs c;
-    c.X16 = X16; c.ldx = ldx; c.x_amax = x_amax; c.y_amax = y_amax; c.m0 = amax_m0; c.m1 = amax_m1;
-    return enqueue_spmm(h, X16, N, nullptr, Y16, st, h->d_acc, h->d_cnt, h->timers_on, &c);
+    c.y_amax = y_amax; c.m0 = amax_m0; c.m1 = amax_m1;
+    // One small kernel quantises the activations once into the handle's buffer; it is launched like
+    // the SpMM kernels, so the SpMM's weight copies start while it runs. (Quantising inside the SpMM's
+    // own staging was measured: every one of the 148 CTAs then pulls the fp16 activations through L2
+    // and converts them -- 5 us more than this at N = 1, 8 to 15 us more at N = 16 and 32.)
+    uint16_t* xs = reinterpret_cast<uint16_t*>(h->d_xq + h->xq_bytes);
+    const cudaError_t e = launch_quantize(static_cast<const uint16_t*>(X16), ldx, N, h->host.K,
+                                          static_cast<const uint32_t*>(x_amax), h->d_xq, xs, st);
+    if (e != cudaSuccess) { h->sticky = e; return US_ERR_CUDA; }
+    return enqueue_spmm(h, h->d_xq, N, xs, Y16, st, h->d_acc, h->d_cnt, h->timers_on, &c);
 }
 
 us_status us_absmax_f16(const void* X16, int64_t ldx, int32_t N, int64_t K, void* amax, void* stream)
 {
-    if (!X16 || !amax || N < 1 || N > 65535 || K < 1 || ldx < K) return US_ERR_INVALID_ARG;
+    if (!X16 || !amax || N < 1 || N > 64 || K < 1 || ldx < K) return US_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(X16) % 2 || reinterpret_cast<uintptr_t>(amax) % 4) return US_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (cudaMemsetAsync(amax, 0, (size_t)N * sizeof(uint32_t), st) != cudaSuccess) { cudaGetLastError(); return US_ERR_CUDA; }
     const int64_t units = (K + 7) / 8;
-    const unsigned gx = (unsigned)std::max<int64_t>(1, std::min<int64_t>(64, (units + 255) / 256));
-    us::us_absmax_f16_kernel<<<dim3(gx, (unsigned)N), 256, 0, st>>>(static_cast<const uint16_t*>(X16), ldx, K,
+    const unsigned gx = (unsigned)std::max<int64_t>(1, std::min<int64_t>(16, (units + 255) / 256));
+    us::us_absmax_f16_kernel<<<dim3(gx, (unsigned)N), 256, 0, st>>>(static_cast<const uint16_t*>(X16), ldx, K, N,
                                                                     static_cast<uint32_t*>(amax));
     if (cudaGetLastError() != cudaSuccess) return US_ERR_CUDA;
     return US_OK;
@@ -632,16 +653,13 @@ us_status us_absmax_f16(const void* X16, int64_t ldx, int32_t N, int64_t K, void
 us_status us_quantize_f16(const void* X16, int64_t ldx, int32_t N, int64_t K, const void* amax, void* Xq,
                           void* x_scale, void* stream)
 {
-    if (!X16 || !amax || !Xq || N < 1 || N > 65535 || K < 1 || ldx < K) return US_ERR_INVALID_ARG;
+    if (!X16 || !amax || !Xq || N < 1 || N > 64 || K < 1 || ldx < K) return US_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(X16) % 2 || reinterpret_cast<uintptr_t>(amax) % 4 ||
         reinterpret_cast<uintptr_t>(x_scale) % 2) return US_ERR_INVALID_ARG;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int64_t units = (K + 7) / 8;
-    const unsigned gx = (unsigned)std::max<int64_t>(1, std::min<int64_t>(64, (units + 255) / 256));
-    us::us_quantize_f16_kernel<<<dim3(gx, (unsigned)N), 256, 0, st>>>(static_cast<const uint16_t*>(X16), ldx, K,
-                                                                      static_cast<const uint32_t*>(amax),
-                                                                      static_cast<uint8_t*>(Xq), static_cast<uint16_t*>(x_scale));
-    if (cudaGetLastError() != cudaSuccess) return US_ERR_CUDA;
+    const cudaError_t e = launch_quantize(static_cast<const uint16_t*>(X16), ldx, N, K, static_cast<const uint32_t*>(amax),
+                                          static_cast<uint8_t*>(Xq), static_cast<uint16_t*>(x_scale),
+                                          static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { cudaGetLastError(); return US_ERR_CUDA; }
     return US_OK;
 }
 

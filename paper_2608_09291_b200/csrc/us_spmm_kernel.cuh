@@ -60,13 +60,9 @@ struct SpmmParams {
     uint32_t slot_bytes;        // ring slot size (max tile blob + slack), multiple of 128
     int32_t x_fast;             // 2: K % 32 == 0 (16-byte loads); 1: K % 8 == 0 (4-byte loads); 0: bytes
     int32_t fp16_out;
-    // Chained call: the activations arrive as fp16 (N rows of ldx16 elements) with the per-token
-    // absmax of the quantised range, and are quantised to INT4 while they are staged; the epilogue
-    // can leave the per-token absmax of output rows [amax_m0, amax_m1) for the next call.
-    const uint16_t* X16;        // nullptr: X holds packed INT4
-    const uint32_t* x_amax;     // N words: fp16 bit pattern of max |x| per token
-    uint32_t* y_amax;           // N words (zero on entry), or nullptr
-    int64_t ldx16;
+    // Chained call: the epilogue leaves the per-token absmax of the fp16 outputs of rows
+    // [amax_m0, amax_m1) in an absmax buffer (layout below) for the quantiser of the next call.
+    uint32_t* y_amax;           // or nullptr
     int32_t amax_m0, amax_m1;
     uint32_t wait_ns_hi;        // bounded waits give up after this many ns >> 10
     uint32_t withhold;          // test hook: position whose copy is never issued (~0u = none)
@@ -327,92 +323,13 @@ __device__ __forceinline__ void stage_x(const SpmmParams& p, int seg0, int n_seg
     }
 }
 
-// ---- per-token symmetric INT4 quantisation of an fp16 activation ------------------------------
-// step s = max(RN_fp16(amax / 7), 2^-24), code = clamp(RNE(y / s), -8, 7); the quotients are IEEE
-// fp32 divisions, so the codes are the same on every implementation of this definition.
-__device__ __forceinline__ float requant_step(uint32_t amax_bits)
-{
-    const float a = __half2float(__ushort_as_half((unsigned short)amax_bits));
-    const float s = __half2float(__float2half_rn(__fdiv_rn(a, 7.0f)));
-    return fmaxf(s, 5.9604644775390625e-08f);
-}
-__device__ __forceinline__ uint32_t requant_code(unsigned short y_bits, float step)
-{
-    const int q = __float2int_rn(__fdiv_rn(__half2float(__ushort_as_half(y_bits)), step));
-    return (uint32_t)max(-8, min(7, q)) & 0xFu;
-}
-// eight fp16 values (four words, element e in half e) -> one word of eight INT4 codes (element e in
-// nibble e): the layout of the packed INT4 input
-__device__ __forceinline__ uint32_t requant8(const uint4 h, float step)
-{
-    const uint32_t w[4] = {h.x, h.y, h.z, h.w};
-    uint32_t v = 0;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        v |= requant_code((unsigned short)(w[i] & 0xFFFFu), step) << (8 * i);
-        v |= requant_code((unsigned short)(w[i] >> 16), step) << (8 * i + 4);
-    }
-    return v;
-}
-
-// X staging of a chained call: as the general path of stage_x, with the eight codes of a unit
-// quantised from fp16 here instead of read packed. Kept out of line: it runs once per K range and
-// must not cost the decode loop registers.
-struct StageF16 {   // by value: taking the address of the kernel's parameter block would copy it to the stack
-    const uint16_t* X16;
-    const uint32_t* x_amax;
-    int64_t ldx16;
-    int32_t K, N, K_L;
-};
-template <int NT, bool XP>
-__device__ __noinline__ void stage_x_f16(const StageF16 p, int seg0, int n_seg, uint8_t* x8, int xstride, int32_t* sx16)
-{
-    const int rows = NT * 8;
-    const int wpr = p.K_L / 8;
-    const int total = rows * n_seg * wpr;
-    const bool vec = (p.ldx16 % 8 == 0) && (reinterpret_cast<uintptr_t>(p.X16) % 16 == 0);
-    constexpr int kBatch = 4;
-    for (int u0 = threadIdx.x; u0 < total; u0 += kBatch * blockDim.x) {
-        uint4 h[kBatch];
-        float step[kBatch];
-#pragma unroll
-        for (int b = 0; b < kBatch; ++b) {
-            const int u = u0 + b * blockDim.x;
-            h[b] = make_uint4(0, 0, 0, 0);
-            step[b] = 1.f;
-            if (u < total) {
-                const int pi = u / wpr, wi = u - pi * wpr;
-                const int sgl = pi / rows, n = pi - sgl * rows;
-                const int64_t k = (int64_t)(seg0 + sgl) * p.K_L + 8 * wi;
-                if (n < p.N && k < p.K) {
-                    const uint16_t* src = p.X16 + (int64_t)n * p.ldx16 + k;
-                    step[b] = requant_step(__ldg(p.x_amax + n));
-                    if (vec && k + 8 <= p.K) {
-                        h[b] = __ldg(reinterpret_cast<const uint4*>(src));
-                    } else {
-                        uint32_t w[4] = {0, 0, 0, 0};
-                        for (int e = 0; e < 8; ++e)
-                            if (k + e < p.K) w[e >> 1] |= (uint32_t)__ldg(src + e) << (16 * (e & 1));
-                        h[b] = make_uint4(w[0], w[1], w[2], w[3]);
-                    }
-                }
-            }
-        }
-#pragma unroll
-        for (int b = 0; b < kBatch; ++b) {
-            const int u = u0 + b * blockDim.x;
-            if (u < total) {
-                const int pi = u / wpr, wi = u - pi * wpr;
-                const int sgl = pi / rows, n = pi - sgl * rows;
-                const uint32_t v = requant8(h[b], step[b]);
-                int32_t s = 0;
-                if (XP) *reinterpret_cast<uint32_t*>(x8 + n * xstride + (sgl * p.K_L + 8 * wi) / 2) = pack8(v, s);
-                else *reinterpret_cast<uint2*>(x8 + n * xstride + sgl * p.K_L + 8 * wi) = expand8(v, s);
-                if (s) atomicAdd(sx16 + pi, s);
-            }
-        }
-    }
-}
+// ---- absmax buffer of a chained call -----------------------------------------------------------
+// kAmaxWords 32-bit words: word 0 = P, the number of parts; part p < P holds, for token n < 64, the
+// fp16 bit pattern of a partial max |y| at word 64 + 64 * p + n. The absmax of a token is the largest
+// of its P words. Every producer writes all of its parts (one per CTA) with plain stores, so the
+// buffer needs no clearing and no atomics.
+constexpr int kAmaxParts = kMaxCtas;
+constexpr int kAmaxWords = 64 * (1 + kAmaxParts);
 
 // Store the 16 x N results held in fragment order in v: fragment rows g -> original row m_lo,
 // rows g + 8 -> m_hi (negative = padding row), with the optional fp16 dequantisation.
@@ -423,7 +340,6 @@ struct StoreCtx {   // what the store needs, by value (the full parameter block 
     int32_t* acc;
     uint32_t* cnt;
     int32_t M, N, fp16_out;
-    const uint32_t* x_amax;     // chained call: the activation scales follow from these
     uint32_t* amax_s;           // shared-memory per-token absmax of the stored fp16 values, or nullptr
     int32_t amax_m0, amax_m1;
 };
@@ -466,7 +382,6 @@ __device__ __forceinline__ void store_rows(const StoreCtx p, const int (&v)[NT][
             if (p.fp16_out) {
                 float sx;
                 if (ScalePre<NT>::kSx && pre && pre->have_sx) sx = __half2float(__ushort_as_half(pre->sx[ScalePre<NT>::kSx ? nt : 0][j & 1]));
-                else if (p.x_amax) sx = requant_step(__ldg(p.x_amax + n));
                 else sx = __half2float(__ushort_as_half(__ldg(p.x_scale + n)));
                 const float r = (float)v[nt][j] * ((j < 2) ? sw_lo : sw_hi) * sx;
                 const __half h = __float2half_rn(r);
@@ -632,7 +547,14 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
     // Programmatic dependent launch: let the next kernel of the stream start its own prologue
     // (parameter fetch, offsets, first weight tiles) while this one is still working.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (beg >= end) return;
+    if (beg >= end) {   // no work: a chained call still owes its part of the absmax buffer
+        if (p.y_amax && threadIdx.x < 64) {
+            asm volatile("griddepcontrol.wait;" ::: "memory");   // the buffer may still be read by the kernel before
+            p.y_amax[64 + 64 * blockIdx.x + threadIdx.x] = 0;
+            if (blockIdx.x == 0 && threadIdx.x == 0) p.y_amax[0] = gridDim.x;
+        }
+        return;
+    }
     if (timing) dbg[0] = clock64() - t_start;
 
     // position u of the processing order -> K range, strip, segment within the range, tile index
@@ -749,7 +671,7 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
     }
     if (timing) dbg[1] = clock64() - t_start;
     if (threadIdx.x == 0) { claim[0] = beg + (uint32_t)n_static * (uint32_t)n_warps * R; claim[1] = 0; }
-    if (threadIdx.x < NT * 8) amax_s[threadIdx.x] = 0;
+    if (threadIdx.x < 64) amax_s[threadIdx.x] = 0;
     // refill slot s with the position fetched ahead
     auto refill = [&](int s) {
         if (lane == 0 && ahead < end && ahead != p.withhold) {
@@ -815,16 +737,14 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
                 const int n = nt * 8 + (lane & 3) * 2 + j;
-                unsigned short sxb = 0;
-                if (n < p.N) sxb = p.x_amax ? __half_as_ushort(__float2half_rn(requant_step(__ldg(p.x_amax + n)))) : __ldg(p.x_scale + n);
-                spre.sx[nt][j] = sxb;
+                spre.sx[nt][j] = n < p.N ? __ldg(p.x_scale + n) : (unsigned short)0;
             }
         spre.have_sx = true;
     }
     const int g_first = (kr_first == n_kr - 1) ? g_last : p.G;   // segments in that range
     constexpr int kXPre = NT <= 4 ? 8 : 0;   // 16-byte units of X a thread prefetches
     const int x_sh = 31 - __clz(p.K_L / 32);   // log2(units per (segment, token)) when a power of two
-    const bool x_early = kXPre > 0 && p.x_fast == 2 && (1 << x_sh) == p.K_L / 32 && p.X16 == nullptr;
+    const bool x_early = kXPre > 0 && p.x_fast == 2 && (1 << x_sh) == p.K_L / 32;
     uint4 xpre[kXPre > 0 ? kXPre : 1];
     const int x_upr = p.K_L / 32, x_total = NT * 8 * g_first * x_upr;
     if (x_early) {
@@ -850,7 +770,7 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
     const uint32_t lut_a = smem_u32(lut) + 4u * (uint32_t)(lane & (p.lut_rep - 1));
 
     const StoreCtx sctx{p.Y, p.w_scale, p.x_scale, p.acc, p.cnt, p.M, p.N, p.fp16_out,
-                        p.x_amax, p.y_amax ? amax_s : nullptr, p.amax_m0, p.amax_m1};
+                        p.y_amax ? amax_s : nullptr, p.amax_m0, p.amax_m1};
     auto store_strip = [&](int rb, int (&v)[NT][4], int m_lo, int m_hi) {
         if (m_lo == kNoRow) {   // not prefetched by the caller
             m_lo = __ldg(p.row_order + rb * 16 + (lane >> 2));
@@ -932,8 +852,6 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
                 }
             }
             stage_x<NT, XP>(p, kr * p.G, g_kr, x8, xstride, sx16, kXPre * (int)blockDim.x);
-        } else if (p.X16) {
-            stage_x_f16<NT, XP>(StageF16{p.X16, p.x_amax, p.ldx16, p.K, p.N, p.K_L}, kr * p.G, g_kr, x8, xstride, sx16);
         } else {
             stage_x<NT, XP>(p, kr * p.G, g_kr, x8, xstride, sx16, 0);
         }
@@ -1102,10 +1020,9 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
             asm volatile("atom.acq_rel.cta.shared.add.u32 %0, [%1], 1;" : "=r"(old) : "r"(smem_u32(claim + 1)) : "memory");
         old = __shfl_sync(0xffffffffu, old, 0);
         if (old == (uint32_t)n_warps - 1u) {
-            for (int n = lane; n < NT * 8 && n < p.N; n += 32) {
-                const uint32_t b = *(volatile uint32_t*)(amax_s + n);
-                if (b) atomicMax(p.y_amax + n, b);
-            }
+            for (int n = lane; n < 64; n += 32)
+                p.y_amax[64 + 64 * blockIdx.x + n] = n < NT * 8 ? *(volatile uint32_t*)(amax_s + n) : 0u;
+            if (blockIdx.x == 0 && lane == 0) p.y_amax[0] = gridDim.x;
         }
     }
     if (timing && lane == 0) {
