@@ -15,7 +15,7 @@
  * Only tests, the smoke check and the bench's cpu-baseline leg may call this file.
  * It shares no code, header, table or constant with the CUDA library.
  *
- * Conventions (readings of the paper where it is silent are listed in the design notes):
+ * Conventions (where the paper is silent, the reading taken is the one stated here):
  *   W  : int8 row-major M x K, values in [-8,7], 0 = pruned.
  *   LT : local tile H_L x K_L, index t = rb * (Kp/K_L) + kb (row-block major); M and K are
  *        zero-padded up to multiples of H_L and K_L.
