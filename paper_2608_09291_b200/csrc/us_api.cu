@@ -252,6 +252,14 @@ cudaError_t launch_st(const us::SpmmParams& p, bool xp, int grid, int block, int
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     const bool la = p.s_local > 0, timed = p.timers != nullptr;
+    if (p.y_amax) {   // chained call (never timed: enqueue_spmm leaves the timers off)
+        if (NT <= 4 && xp && la) {
+            constexpr int NP = NT <= 4 ? NT : 4;
+            return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NP, ST, true, false, true, true>, p);
+        }
+        return la ? cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, ST, true, false, false, true>, p)
+                  : cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, ST, false, false, false, true>, p);
+    }
     if (NT <= 4 && xp && la) {   // packed X: planned for these classes and local mode only
         constexpr int NP = NT <= 4 ? NT : 4;
         return timed ? cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NP, ST, true, true, true>, p)
@@ -279,6 +287,10 @@ cudaError_t enable_large_smem_st(int bytes)
     if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, ST, false, false>, attr, bytes);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, ST, true, true>, attr, bytes);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, ST, false, true>, attr, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, ST, true, false, false, true>, attr, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, ST, false, false, false, true>, attr, bytes);
+    constexpr int NP = NT <= 4 ? NT : 4;   // packed-X kernels exist for N <= 32
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NP, ST, true, false, true, true>, attr, bytes);
     return e;
 }
 template <int NT>
@@ -376,7 +388,7 @@ us_status enqueue_spmm(us_handle* h, const void* X, int32_t N, const void* x_sca
     p.X = static_cast<const uint8_t*>(X);
     p.x_scale = static_cast<const uint16_t*>(x_scale);
     p.Y = Y; p.acc = acc; p.cnt = cnt; p.err = h->d_err;
-    p.timers = timers ? h->d_timers : nullptr;
+    p.timers = (timers && !(chain && chain->y_amax)) ? h->d_timers : nullptr;
     p.M = (int32_t)hm.M; p.K = (int32_t)hm.K; p.N = N;
     p.n_strips = (int32_t)hm.n_strips; p.n_segs = (int32_t)hm.n_segs;
     p.mask_rows = hm.mask_rows; p.K_L = hm.fmt.K_L;

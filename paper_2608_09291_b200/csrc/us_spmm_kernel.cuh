@@ -354,7 +354,8 @@ struct ScalePre {
     bool have_sx = false;
     unsigned short sx[kSx ? NT : 1][2];
 };
-template <int NT>
+// AM: also track the per-token absmax of the stored fp16 values (chained calls).
+template <int NT, bool AM>
 __device__ __forceinline__ void store_rows(const StoreCtx p, const int (&v)[NT][4], int lane, int m_lo, int m_hi,
                                            const ScalePre<NT>* pre = nullptr, int rb = -2)
 {
@@ -369,7 +370,7 @@ __device__ __forceinline__ void store_rows(const StoreCtx p, const int (&v)[NT][
             if (m_hi >= 0) sw_hi = __half2float(__ushort_as_half(__ldg(p.w_scale + m_hi)));
         }
     }
-    const bool track = p.amax_s != nullptr;
+    constexpr bool track = AM;
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
         uint32_t big[2] = {0u, 0u};   // absmax (fp16 bits) of this lane's stored values of tokens t2, t2 + 1
@@ -478,7 +479,7 @@ __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, ui
 // Last arrival of a strip in the global workspace: read the sums, leave workspace and counter
 // zeroed, dequantise and store. Kept out of line: it runs once per strip at most, and the decode
 // loop's code should stay small enough for the instruction cache.
-template <int NT>
+template <int NT, bool AM>
 __device__ __noinline__ void finalize_strip(const StoreCtx p, int rb, int lane, int m_lo, int m_hi)
 {
     int32_t* accp = p.acc + (size_t)rb * (NT * 128) + lane;
@@ -491,7 +492,7 @@ __device__ __noinline__ void finalize_strip(const StoreCtx p, int rb, int lane, 
             __stcg(accp + nt * 128 + j * 32, 0);
         }
     if (lane == 0) p.cnt[rb] = 0;
-    store_rows<NT>(p, v, lane, m_lo, m_hi);
+    store_rows<NT, AM>(p, v, lane, m_lo, m_hi);
 }
 
 // ---- the kernel -----------------------------------------------------------------------------
@@ -512,7 +513,9 @@ constexpr int kTimerWords = kWarpRec * kMaxWarpsPerCta * kMaxCtas;
 // LA = local mode (shared-memory strip accumulators), else direct mode.
 // TIMED = record the diagnostic stage timers (a separate instantiation, so that the production
 // kernel carries none of their clock reads and branches).
-template <int NT, int STAGES, bool LA, bool TIMED, bool XP = false>
+// AM = chained call that leaves the per-token absmax of its fp16 output (separate too: the plain
+// fp16 store measured 2.5 % slower with the tracking compiled in behind a run-time flag).
+template <int NT, int STAGES, bool LA, bool TIMED, bool XP = false, bool AM = false>
 __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -548,7 +551,7 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
     // (parameter fetch, offsets, first weight tiles) while this one is still working.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (beg >= end) {   // no work: a chained call still owes its part of the absmax buffer
-        if (p.y_amax && threadIdx.x < 64) {
+        if (AM && threadIdx.x < 64) {
             asm volatile("griddepcontrol.wait;" ::: "memory");   // the buffer may still be read by the kernel before
             p.y_amax[64 + 64 * blockIdx.x + threadIdx.x] = 0;
             if (blockIdx.x == 0 && threadIdx.x == 0) p.y_amax[0] = gridDim.x;
@@ -671,7 +674,7 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
     }
     if (timing) dbg[1] = clock64() - t_start;
     if (threadIdx.x == 0) { claim[0] = beg + (uint32_t)n_static * (uint32_t)n_warps * R; claim[1] = 0; }
-    if (threadIdx.x < 64) amax_s[threadIdx.x] = 0;
+    if (AM && threadIdx.x < 64) amax_s[threadIdx.x] = 0;
     // refill slot s with the position fetched ahead
     auto refill = [&](int s) {
         if (lane == 0 && ahead < end && ahead != p.withhold) {
@@ -770,13 +773,13 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
     const uint32_t lut_a = smem_u32(lut) + 4u * (uint32_t)(lane & (p.lut_rep - 1));
 
     const StoreCtx sctx{p.Y, p.w_scale, p.x_scale, p.acc, p.cnt, p.M, p.N, p.fp16_out,
-                        p.y_amax ? amax_s : nullptr, p.amax_m0, p.amax_m1};
+                        AM ? amax_s : nullptr, p.amax_m0, p.amax_m1};
     auto store_strip = [&](int rb, int (&v)[NT][4], int m_lo, int m_hi) {
         if (m_lo == kNoRow) {   // not prefetched by the caller
             m_lo = __ldg(p.row_order + rb * 16 + (lane >> 2));
             m_hi = __ldg(p.row_order + rb * 16 + (lane >> 2) + 8);
         }
-        store_rows<NT>(sctx, v, lane, m_lo, m_hi, kPreScales ? &spre : nullptr, rb);
+        store_rows<NT, AM>(sctx, v, lane, m_lo, m_hi, kPreScales ? &spre : nullptr, rb);
     };
     // add v to the global workspace of strip rb
     auto red_global = [&](int rb, int (&v)[NT][4]) {
@@ -804,7 +807,7 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
                 m_lo = __ldg(p.row_order + rb * 16 + (lane >> 2));
                 m_hi = __ldg(p.row_order + rb * 16 + (lane >> 2) + 8);
             }
-            finalize_strip<NT>(sctx, rb, lane, m_lo, m_hi);
+            finalize_strip<NT, AM>(sctx, rb, lane, m_lo, m_hi);
         }
     };
 
@@ -1013,7 +1016,7 @@ __global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
         }
     }
     // Chained call: the last warp of the CTA to finish publishes the CTA's per-token absmax.
-    if (p.y_amax) {
+    if (AM) {
         __syncwarp();
         uint32_t old = 0;
         if (lane == 0)
