@@ -56,7 +56,8 @@ int env_int(const char* name, int fallback)
 }
 int pdl_knob() { static int v = env_int("US_PDL", 1); return v; }          // programmatic dependent launch
 int stages_knob() { static int v = env_int("US_STAGES", 0); return v; }    // ring slots per warp, 0 = automatic
-int max_warps() { static int v = std::min(16, std::max(2, env_int("US_MAX_WARPS", 16))); return v; }
+// (up to 20 for the N <= 8 kernels; the other kernels are compiled for 16)
+int max_warps() { static int v = std::min(20, std::max(2, env_int("US_MAX_WARPS", 16))); return v; }
 int coresident_knob() { static int v = env_int("US_CORESIDENT", 1); return v; }  // small problems: half an SM per CTA
 constexpr int kLocalAccBudget = 32 * 1024;   // local strip sums a K-range width is chosen with
 constexpr int kLocalAccCap = 48 * 1024;      // ... and what is taken if nothing fits that
@@ -120,7 +121,7 @@ bool plan_launch(const us_handle* h, int N, LaunchGeom* g)
     // warp and more warps -- measured on the 70B-shaped FFN: 16 warps x 1 slot beat 9 warps x 2.
     auto warps_for = [&](int stages) {
         const int fixed = fixed_base + 32 * stages * 8;
-        return std::min((limit - fixed) / (int)(stages * g->slot_bytes), max_warps());
+        return std::min((limit - fixed) / (int)(stages * g->slot_bytes), g->nt == 1 ? max_warps() : std::min(16, max_warps()));
     };
     {
         const int w32 = std::max(warps_for(1), warps_for(2));
@@ -150,7 +151,7 @@ bool plan_launch(const us_handle* h, int N, LaunchGeom* g)
     if (coresident_knob() && co_class && per_cta <= kCoresidentTiles && stages_knob() == 0) {
         const int half = 228 * 1024 / 2 - 1024 - 512;   // per SM: 228 KB, 1 KB reserved per CTA
         const int fixed8 = fixed_for(8) + 32 * 8;
-        int w = std::min(g->nt == 1 ? h->co_warps : h->co_warps2, max_warps());
+        int w = std::min(g->nt == 1 ? h->co_warps : h->co_warps2, g->nt == 1 ? max_warps() : std::min(16, max_warps()));
         while (w >= 8 && fixed8 + w * (int)g->slot_bytes > half) --w;
         if (w >= 8) { stages = 1; lut_rep = 8; warps = w; fixed = fixed8; }
     }

@@ -507,7 +507,7 @@ __device__ __forceinline__ uint32_t fdiv(uint32_t u, unsigned long long m)
 // before the first tile, [6] start ns, [7] activations staged ns, [8] end ns, [9..12] prologue
 // checkpoints (cycles: range known, copies issued, table done, X staged), [13] ns past the
 // dependency wait.
-constexpr int kWarpRec = 16, kMaxWarpsPerCta = 16;
+constexpr int kWarpRec = 16, kMaxWarpsPerCta = 24;
 constexpr int kTimerWords = kWarpRec * kMaxWarpsPerCta * kMaxCtas;
 
 // LA = local mode (shared-memory strip accumulators), else direct mode.
@@ -516,7 +516,9 @@ constexpr int kTimerWords = kWarpRec * kMaxWarpsPerCta * kMaxCtas;
 // AM = chained call that leaves the per-token absmax of its fp16 output (separate too: the plain
 // fp16 store measured 2.5 % slower with the tracking compiled in behind a run-time flag).
 template <int NT, int STAGES, bool LA, bool TIMED, bool XP = false, bool AM = false>
-__global__ void __launch_bounds__(512, 1) us_spmm_kernel(const SpmmParams p)
+// (N <= 8 kernels are compiled for up to 20 warps: 80 registers instead of 90, which lets 12 instead of 10 warps of
+// two half-SM CTAs share an SM; more than 16 warps per full-SM CTA were measured and do not pay.)
+__global__ void __launch_bounds__(NT == 1 ? 640 : 512, 1) us_spmm_kernel(const SpmmParams p)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
