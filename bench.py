@@ -480,8 +480,8 @@ def kernel_label(binding, handle, N):
 
 # Measured DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch, from the ncu
 # captures of the same kernel build (one launch each; commands in the capture summaries).
-TRAFFIC_BYTES_PER_LAUNCH = 8_202_752          # 4096x4096, s = 0.5, N = 8, fp16: 8.2028 MB read, 0 written
-TRAFFIC_BYTES_PER_LAUNCH_LARGE = 102_230_784  # 28672x8192, s = 0.6, N = 8, int32: 98.02 MB read + 4.21 MB written
+TRAFFIC_BYTES_PER_LAUNCH = 8_200_960          # 4096x4096, s = 0.5, N = 8, fp16: 8.2010 MB read, 0 written
+TRAFFIC_BYTES_PER_LAUNCH_LARGE = 102_112_256  # 28672x8192, s = 0.6, N = 8, int32: 98.01 MB read + 4.10 MB written
 
 
 def sweep(binding, torch, workloads, l2, peak_gbs):
