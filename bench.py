@@ -10,7 +10,7 @@ row-varying density; the 13B-shaped decoder layer; the 70B-shaped FFN N sweep) a
 same line under "sweep".
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-sweep]
-  python bench.py --only M,K,s,N[,int32|fp16[,K_L[,N_max]]]     one case with the kernel's stage
+  python bench.py --only M,K,s,N[,int32|fp16[,K_L[,N_max[,q4]]]]     one case with the kernel's stage
                                                                timers (the command of the ncu captures)
 
 With --gpus N > 1 and no torchrun environment the script starts itself N times under
@@ -487,7 +487,9 @@ TRAFFIC_BYTES_PER_LAUNCH_LARGE = 102_112_256  # 28672x8192, s = 0.6, N = 8, int3
 def sweep(binding, torch, workloads, l2, peak_gbs):
     rows = []
 
-    def run_case(name, M, K, s, seed, Ns, outs, row_varying=False, flags=0):
+    def run_case(name, M, K, s, seed, Ns, outs, row_varying=False, flags=0, q4=False):
+        """q4: the folded format (16, K_L, 2, 2) -- one mask bit per 2 x 2 weights -- at the K_L the
+        library picks for this shape, instead of the default (16, K_L, 2, 1)."""
         W = workloads.make_weight(M, K, s, seed, row_varying)
         Nmax = max(Ns)
         X = workloads.make_x(K, Nmax, seed)
@@ -495,8 +497,14 @@ def sweep(binding, torch, workloads, l2, peak_gbs):
         probe = binding.us_encode(W, None, None, Nmax, binding.US_ENCODE_HOST_ONLY | flags)
         st = binding.us_get_stats(probe)
         binding.us_destroy(probe)
+        fmt = None
+        if q4:
+            fmt = (16, st["fmt"][1], 2, 2)
+            probe = binding.us_encode(W, None, fmt, Nmax, binding.US_ENCODE_HOST_ONLY | flags)
+            st = binding.us_get_stats(probe)
+            binding.us_destroy(probe)
         R = replicas_for(st, l2)
-        case = Case(binding, torch, W, s_w, X, s_x, Nmax, R, flags=flags)
+        case = Case(binding, torch, W, s_w, X, s_x, Nmax, R, fmt=fmt, flags=flags)
         for fp16 in outs:
             for N in Ns:
                 passes = max(3, int(2e-2 / max(1e-6, 3e-6 * R)))
@@ -512,7 +520,8 @@ def sweep(binding, torch, workloads, l2, peak_gbs):
                              "bytes_q1": q1, "pct_of_8tbs_on_q1_bytes": 100 * q1 / t / 1e9 / CONTRACT_PEAK_GBS,
                              "bytes_dense_int4": dn, "us_dense_int4_at_8tbs": dn / CONTRACT_PEAK_GBS / 1e3,
                              "dense_equiv_tops": 2.0 * M * K * N / t / 1e12, "replicas": R,
-                             "pmr": case.stats["pmr"], "kernel": kernel_label(binding, case.sw[0].handle, N)})
+                             "pmr": case.stats["pmr"], "format": list(case.stats["fmt"]),
+                             "kernel": kernel_label(binding, case.sw[0].handle, N)})
         case.close()
         del case
         torch.cuda.empty_cache()
@@ -530,6 +539,14 @@ def sweep(binding, torch, workloads, l2, peak_gbs):
     # Bitmap-aware row pairing inside each strip (the per-strip form of Alg. 1): fewer union bits.
     run_case("attn7b_paired", 4096, 4096, 0.5, 201, [8], [True], flags=binding.US_ENCODE_PAIR_ROWS)
     run_case("ffn70b_up_paired", 28672, 8192, 0.6, 500, [8], [False], flags=binding.US_ENCODE_PAIR_ROWS)
+    # The paper's 2 x 2 union mask (Q = 4) in the folded kernel layout, N <= 8: more bytes, fewer decode
+    # instructions per weight. Same matrices and seeds as the rows above.
+    for i, s in enumerate((0.3, 0.5, 0.7)):
+        run_case("attn7b_q4", 4096, 4096, s, 200 + i, [1, 8], [True], q4=True)
+    run_case("ffn7b_up_q4", 11008, 4096, 0.5, 300, [8], [True], row_varying=True, flags=SORT, q4=True)
+    run_case("ffn7b_down_q4", 4096, 11008, 0.5, 302, [8], [True], row_varying=True, flags=SORT, q4=True)
+    run_case("ffn70b_up_q4", 28672, 8192, 0.6, 500, [1, 8], [False], q4=True)
+    run_case("ffn70b_down_q4", 8192, 28672, 0.6, 501, [1, 8], [False], q4=True)
     for s in (0.3, 0.5, 0.7):                                                                  # config 4
         rows.append(layer_chain(binding, torch, workloads, l2, s))
         rows.append(layer_chain_requant(binding, torch, workloads, l2, s))
@@ -695,7 +712,8 @@ def run_only(args):
     f = args.only.split(",")
     M, K, s, N = int(f[0]), int(f[1]), float(f[2]), int(f[3])
     fp16 = len(f) > 4 and f[4] == "fp16"
-    fmt = (16, int(f[5]), 2, 1) if len(f) > 5 and int(f[5]) > 0 else None
+    # K_L > 0 picks the tile width; a seventh field "q4" the folded format (16, K_L, 2, 2)
+    fmt = (16, int(f[5]), 2, 2 if (len(f) > 7 and f[7] == "q4") else 1) if len(f) > 5 and int(f[5]) > 0 else None
     n_max = int(f[6]) if len(f) > 6 else N   # largest N the handles are encoded for
     torch.cuda.set_device(0)
     l2 = torch.cuda.get_device_properties(0).L2_cache_size or L2_BYTES_FALLBACK
@@ -774,7 +792,7 @@ def main(argv=None):
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-sweep", action="store_true")
-    ap.add_argument("--only", default=None, metavar="M,K,s,N[,int32|fp16[,K_L[,N_max]]]",
+    ap.add_argument("--only", default=None, metavar="M,K,s,N[,int32|fp16[,K_L[,N_max[,q4]]]]",
                     help="time one case only, with the kernel's stage timers: the small run of the ncu captures")
     ap.add_argument("--chain", action="store_true",
                     help="time only the 13B-shaped layer, as seven plain calls and as a chain of four chained calls")

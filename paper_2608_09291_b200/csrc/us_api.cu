@@ -20,6 +20,7 @@ struct us_handle {
     int max_smem = 0;
     int co_warps = 10;   // warps of an N <= 8 CTA when two CTAs share an SM's registers
     int co_warps2 = 8;   // the same for the N = 9..16 kernel with packed activations
+    int co_warps_fold = 8;   // the same for the folded-tile (two column areas) N <= 8 kernel
     uint8_t* d_blob = nullptr;
     uint32_t* d_item_off = nullptr;
     std::vector<uint32_t> cta_begin[4];  // schedule per N class (NT = 1, 2, 4, 8)
@@ -77,6 +78,13 @@ struct LaunchGeom {
 // 16 warps and two ranges by 25 % on a 13824 x 5120 matrix at N = 16).
 // Shared memory of one K range's activations: int8 (one byte per token and k, 32 bytes of pad per
 // token row) or packed (half of that).
+// Ring slot: the largest tile plus the two payload rows the decode's window loads may read past a
+// stream's end (rows are 128 bytes per column area).
+uint32_t slot_bytes_for(const us::HostMatrix& hm)
+{
+    return (hm.max_item_bytes + 256u * (uint32_t)hm.fmt.C_A + 127u) & ~127u;
+}
+
 int64_t x_bytes(int nt, int64_t G, int K_L, bool xp)
 {
     return xp ? (int64_t)nt * 8 * (G * K_L / 2 + 16) : (int64_t)nt * 8 * (G * K_L + 32);
@@ -85,7 +93,7 @@ int64_t x_bytes(int nt, int64_t G, int K_L, bool xp)
 int segs_per_range(const us::HostMatrix& hm, int nt, int limit, int64_t min_ranges, bool xp)
 {
     const int64_t n_segs = hm.n_segs;
-    const int slot = (int)((hm.max_item_bytes + 256u + 127u) & ~127u);
+    const int slot = (int)slot_bytes_for(hm);
     const int acc = nt * 512 * 2 <= kLocalAccBudget ? kLocalAccBudget : 0;
     const int other = 256 * 8 * 4 + (int)us::kLutScratchBytes + acc + 2 * us::kOffTable * 4 + 1280;
     for (int64_t r = std::max<int64_t>(1, min_ranges); r <= n_segs; ++r) {
@@ -108,7 +116,7 @@ bool plan_launch(const us_handle* h, int N, LaunchGeom* g)
     g->cls = class_of(g->nt);
     const int G = h->G[g->cls], s_local = h->s_local[g->cls];
     g->xp = h->xp[g->cls];
-    g->slot_bytes = (h->host.max_item_bytes + 256u + 127u) & ~127u;
+    g->slot_bytes = slot_bytes_for(h->host);
     // selector table copies: 32 (conflict-free lookups) when that costs no warp, else 8
     int lut_rep = 32;
     auto fixed_for = [&](int rep) {
@@ -121,7 +129,8 @@ bool plan_launch(const us_handle* h, int N, LaunchGeom* g)
     // warp and more warps -- measured on the 70B-shaped FFN: 16 warps x 1 slot beat 9 warps x 2.
     auto warps_for = [&](int stages) {
         const int fixed = fixed_base + 32 * stages * 8;
-        return std::min((limit - fixed) / (int)(stages * g->slot_bytes), g->nt == 1 ? max_warps() : std::min(16, max_warps()));
+        return std::min((limit - fixed) / (int)(stages * g->slot_bytes),
+                        (g->nt == 1 && h->host.fmt.C_A == 1) ? max_warps() : std::min(16, max_warps()));
     };
     {
         const int w32 = std::max(warps_for(1), warps_for(2));
@@ -151,7 +160,9 @@ bool plan_launch(const us_handle* h, int N, LaunchGeom* g)
     if (coresident_knob() && co_class && per_cta <= kCoresidentTiles && stages_knob() == 0) {
         const int half = 228 * 1024 / 2 - 1024 - 512;   // per SM: 228 KB, 1 KB reserved per CTA
         const int fixed8 = fixed_for(8) + 32 * 8;
-        int w = std::min(g->nt == 1 ? h->co_warps : h->co_warps2, g->nt == 1 ? max_warps() : std::min(16, max_warps()));
+        const bool fold = h->host.fmt.C_A == 2;
+        int w = std::min(g->nt == 1 ? (fold ? h->co_warps_fold : h->co_warps) : h->co_warps2,
+                         (g->nt == 1 && !fold) ? max_warps() : std::min(16, max_warps()));
         while (w >= 8 && fixed8 + w * (int)g->slot_bytes > half) --w;
         if (w >= 8) { stages = 1; lut_rep = 8; warps = w; fixed = fixed8; }
     }
@@ -188,7 +199,7 @@ void plan_classes(us_handle* h, int n_cta, std::vector<uint32_t> (&sched)[4])
                     const int need = worst * nt * 512;
                     if (pass == 0 && need <= kLocalAccBudget) { *s_local = worst; return G; }
                     if (pass == 1 && need <= kLocalAccCap) {
-                        const int slot = (int)((h->host.max_item_bytes + 256u + 127u) & ~127u);
+                        const int slot = (int)slot_bytes_for(h->host);
                         const int64_t fixed = 256 * 8 * 4 + (int64_t)us::kLutScratchBytes + need + 2 * us::kOffTable * 4 + 1280 +
                                               x_bytes(nt, G, h->host.fmt.K_L, xp) + (int64_t)G * nt * 32;
                         if ((limit - fixed) / slot >= 11) { *s_local = worst; return G; }
@@ -211,7 +222,7 @@ void plan_classes(us_handle* h, int n_cta, std::vector<uint32_t> (&sched)[4])
         // ranges become one); 5120 x 5120 12.0 -> 9.4 us (one range either way, but a CTA's share is
         // small and the staging pass and the freed shared memory count for more than the decode);
         // 13824 x 5120 15.7 -> 16.0 us (one range either way, long decode): not taken there.
-        if (nt <= 4) {
+        if (nt <= 4 && h->host.fmt.C_A == 1) {   // (no packed-X kernel for folded tiles)
             const int64_t n_segs = h->host.n_segs;
             const int64_t ranges = h->s_local[c] > 0 ? (n_segs + h->G[c] - 1) / h->G[c] : n_segs + 1;
             const bool small_share = nt >= 2 && (int64_t)h->host.blob.size() / std::max(1, n_cta) < 128 * 1024;
@@ -253,6 +264,12 @@ cudaError_t launch_st(const us::SpmmParams& p, bool xp, int grid, int block, int
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     const bool la = p.s_local > 0, timed = p.timers != nullptr;
+    if (p.fold_kb) {   // folded tiles (two column areas): N <= 8 kernels only, checked by the caller
+        if (la) return timed ? cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<1, ST, true, true, false, false, 2>, p)
+                             : cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<1, ST, true, false, false, false, 2>, p);
+        return timed ? cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<1, ST, false, true, false, false, 2>, p)
+                     : cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<1, ST, false, false, false, false, 2>, p);
+    }
     if (p.y_amax) {   // chained call (never timed: enqueue_spmm leaves the timers off)
         if (NT <= 4 && xp && la) {
             constexpr int NP = NT <= 4 ? NT : 4;
@@ -292,6 +309,12 @@ cudaError_t enable_large_smem_st(int bytes)
     if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, ST, false, false, false, true>, attr, bytes);
     constexpr int NP = NT <= 4 ? NT : 4;   // packed-X kernels exist for N <= 32
     if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NP, ST, true, false, true, true>, attr, bytes);
+    if (NT == 1) {   // folded tiles
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<1, ST, true, false, false, false, 2>, attr, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<1, ST, false, false, false, false, 2>, attr, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<1, ST, true, true, false, false, 2>, attr, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<1, ST, false, true, false, false, 2>, attr, bytes);
+    }
     return e;
 }
 template <int NT>
@@ -393,6 +416,7 @@ us_status enqueue_spmm(us_handle* h, const void* X, int32_t N, const void* x_sca
     p.M = (int32_t)hm.M; p.K = (int32_t)hm.K; p.N = N;
     p.n_strips = (int32_t)hm.n_strips; p.n_segs = (int32_t)hm.n_segs;
     p.mask_rows = hm.mask_rows; p.K_L = hm.fmt.K_L;
+    p.fold_kb = hm.fmt.C_A == 2 ? hm.nkb / 2 : 0;
     p.slot_bytes = g.slot_bytes;
     p.x_fast = (hm.K % 32 == 0) ? 2 : (hm.K % 8 == 0) ? 1 : 0;
     p.fp16_out = x_scale ? 1 : 0;
@@ -451,6 +475,8 @@ us_status us_encode(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_sca
         *out = h;
         return US_OK;
     }
+    // folded tiles (two column areas): kernels for N <= 8 only
+    if (hm.fmt.C_A == 2 && max_N > 8 && !host_only) { delete h; return US_ERR_UNSUPPORTED; }
     // the kernel's index arithmetic (exact division by multiplication) needs u * d < 2^40 for every
     // position u < n_items and divisor d <= n_items
     if (hm.n_items >= (1 << 20) || hm.n_segs >= (1 << 16)) {
@@ -479,6 +505,8 @@ us_status us_encode(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_sca
         cudaFuncAttributes fa2;
         if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa2, (const void*)us::us_spmm_kernel<2, 1, true, false, true>);
         if (e == cudaSuccess) h->co_warps2 = 32768 / (32 * ((fa2.numRegs + 7) / 8 * 8));
+        if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa2, (const void*)us::us_spmm_kernel<1, 1, true, false, false, false, 2>);
+        if (e == cudaSuccess) h->co_warps_fold = 32768 / (32 * ((fa2.numRegs + 7) / 8 * 8));
     }
     if (e != cudaSuccess) { delete h; return US_ERR_CUDA; }
 
@@ -628,6 +656,7 @@ us_status us_spmm_requant(us_handle* h, const void* X16, int64_t ldx, const void
     if (!h || !X16 || !x_amax || !Y16 || N < 1 || N > h->max_N) return US_ERR_INVALID_ARG;
     if (!h->on_device) return US_ERR_UNSUPPORTED;
     if (!h->d_w_scale) return US_ERR_INVALID_ARG;   // fp16 output needs the weight scales
+    if (y_amax && h->host.fmt.C_A != 1) return US_ERR_UNSUPPORTED;   // no absmax-tracking kernel for folded tiles
     if (ldx < h->host.K) return US_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(X16) % 2 || reinterpret_cast<uintptr_t>(Y16) % 2 ||
         reinterpret_cast<uintptr_t>(x_amax) % 4 || reinterpret_cast<uintptr_t>(y_amax) % 4) return US_ERR_INVALID_ARG;

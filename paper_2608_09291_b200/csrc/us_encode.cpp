@@ -234,7 +234,8 @@ us_status encode_host(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_s
     HostMatrix& h = *out;
     h = HostMatrix();
     h.M = M; h.K = K; h.fmt = fmt;
-    h.kernel_layout = fmt.H_L == 16 && fmt.R_A == 2 && fmt.C_A == 1 && fmt.K_L % 128 == 0 && fmt.K_L <= 8192;
+    h.kernel_layout = fmt.H_L == 16 && fmt.R_A == 2 && fmt.K_L <= 8192 &&
+                      ((fmt.C_A == 1 && fmt.K_L % 128 == 0) || (fmt.C_A == 2 && fmt.K_L % 256 == 0));
     if (!h.kernel_layout) {
         // a valid IE-BME format without a kernel: the paper's arrays, for statistics and decoding
         if (!(flags & US_ENCODE_HOST_ONLY)) return US_ERR_UNSUPPORTED;
@@ -248,7 +249,9 @@ us_status encode_host(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_s
     h.Mp = (M + 15) / 16 * 16;
     h.Kp = (K + fmt.K_L - 1) / fmt.K_L * fmt.K_L;
     h.nkb = fmt.K_L / 32;
-    h.mask_rows = h.nkb / 4;
+    h.mask_rows = h.nkb / (4 * fmt.C_A);
+    // the pairing cost below is written for one column area
+    if (fmt.C_A == 2 && (flags & US_ENCODE_PAIR_ROWS)) { h = HostMatrix(); return US_ERR_UNSUPPORTED; }
     h.n_strips = h.Mp / 16;
     h.n_segs = h.Kp / fmt.K_L;
     h.n_items = h.n_strips * h.n_segs;
@@ -276,7 +279,8 @@ us_status encode_host(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_s
     if (flags & US_ENCODE_PAIR_ROWS) pair_rows(W, M, K, threads, &h);
 
     // ---- build every tile blob (parallel over strips) ------------------------------------
-    const int K_L = fmt.K_L, nkb = h.nkb, mask_rows = h.mask_rows;
+    const int K_L = fmt.K_L, CA = fmt.C_A, nkb = h.nkb / CA, mask_rows = h.mask_rows;   // nkb: mask bytes per lane
+    const int K_B = K_L / CA;                                                            // columns per column area
     const int64_t mask_bytes = (int64_t)mask_rows * 128;
     std::vector<std::vector<uint8_t>> blobs(h.n_items);
     std::atomic<int64_t> nnz{0}, sum_P{0};
@@ -287,7 +291,8 @@ us_status encode_host(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_s
             int32_t o = h.row_order[rb * 16 + r];
             rows[r] = o < 0 ? nullptr : W + (int64_t)o * K;
         }
-        std::vector<uint8_t> stream((size_t)32 * nkb * 8);  // lane-major payload bytes
+        std::vector<uint8_t> stream((size_t)32 * nkb * 8);  // lane-major payload bytes (column area 0)
+        std::vector<uint8_t> stream2(CA == 2 ? (size_t)32 * nkb * 8 : 0);   // column area 1
         std::vector<uint8_t> mask((size_t)32 * nkb);        // lane-major mask bytes
         int len[32];
         int64_t my_nnz = 0, my_P = 0;
@@ -298,30 +303,49 @@ us_status encode_host(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_s
             for (int g = 0; g < 8; ++g) {
                 const int8_t* pa = rows[g];
                 const int8_t* pb = rows[g + 8];
-                const int64_t kend = std::min<int64_t>(K, k0 + K_L);
-                for (int64_t k = k0; k < kend; ++k) {
-                    int lo = pa ? pa[k] : 0, hi = pb ? pb[k] : 0;
-                    if (!(lo | hi)) continue;
-                    if (lo < -8 || lo > 7 || hi < -8 || hi > 7) { bad.store(1); continue; }
-                    my_nnz += (lo != 0) + (hi != 0);
-                    const int kk = (int)(k - k0), kb = kk >> 5, t = (kk >> 3) & 3, j = kk & 7;
+                // kk = column within the column area; with C_A = 2 one mask bit covers columns kk and
+                // kk + K_B of the tile (rows g and g + 8 of each), and the two columns' bytes go to two
+                // streams of equal length
+                for (int kk = 0; kk < K_B; ++kk) {
+                    int v[2][2];   // [column area][row half]
+                    int any = 0;
+                    for (int ca = 0; ca < CA; ++ca) {
+                        const int64_t k = k0 + kk + (int64_t)ca * K_B;
+                        v[ca][0] = (pa && k < K) ? pa[k] : 0;
+                        v[ca][1] = (pb && k < K) ? pb[k] : 0;
+                        any |= v[ca][0] | v[ca][1];
+                    }
+                    if (!any) continue;
+                    bool range_ok = true;
+                    for (int ca = 0; ca < CA; ++ca)
+                        for (int r = 0; r < 2; ++r) range_ok = range_ok && v[ca][r] >= -8 && v[ca][r] <= 7;
+                    if (!range_ok) { bad.store(1); continue; }
+                    for (int ca = 0; ca < CA; ++ca) my_nnz += (v[ca][0] != 0) + (v[ca][1] != 0);
+                    const int kb = kk >> 5, t = (kk >> 3) & 3, j = kk & 7;
                     const int lane = 4 * g + t;
                     mask[(size_t)lane * nkb + kb] |= (uint8_t)(1u << j);
-                    stream[(size_t)lane * nkb * 8 + len[lane]++] =
-                        (uint8_t)(((hi & 0xF) << 4) | ((lo + 8) & 0xF));
+                    const size_t at = (size_t)lane * nkb * 8 + len[lane]++;
+                    stream[at] = (uint8_t)(((v[0][1] & 0xF) << 4) | ((v[0][0] + 8) & 0xF));
+                    if (CA == 2) stream2[at] = (uint8_t)(((v[1][1] & 0xF) << 4) | ((v[1][0] + 8) & 0xF));
                 }
             }
             int maxlen = 0;
             for (int l = 0; l < 32; ++l) { maxlen = std::max(maxlen, len[l]); my_P += len[l]; }
             const int J = (maxlen + 3) / 4;
             std::vector<uint8_t>& b = blobs[rb * h.n_segs + sg];
-            b.assign((size_t)mask_bytes + (size_t)J * 128, 0);
+            // payload rows of 32 lane words; with C_A = 2 the rows of the two streams alternate
+            b.assign((size_t)mask_bytes + (size_t)J * 128 * CA, 0);
             for (int l = 0; l < 32; ++l) {
                 for (int w = 0; w < mask_rows; ++w)
                     std::memcpy(&b[(size_t)w * 128 + l * 4], &mask[(size_t)l * nkb + 4 * w], 4);
                 const uint8_t* s = &stream[(size_t)l * nkb * 8];
                 for (int i = 0; i < len[l]; ++i)
-                    b[(size_t)mask_bytes + (size_t)(i >> 2) * 128 + l * 4 + (i & 3)] = s[i];
+                    b[(size_t)mask_bytes + (size_t)(i >> 2) * 128 * CA + l * 4 + (i & 3)] = s[i];
+                if (CA == 2) {
+                    const uint8_t* s2 = &stream2[(size_t)l * nkb * 8];
+                    for (int i = 0; i < len[l]; ++i)
+                        b[(size_t)mask_bytes + (size_t)(i >> 2) * 256 + 128 + l * 4 + (i & 3)] = s2[i];
+                }
             }
         }
         nnz += my_nnz;
@@ -359,7 +383,7 @@ void decode_host(const HostMatrix& h, int8_t* W_out)
 {
     std::memset(W_out, 0, (size_t)(h.M * h.K));
     if (!h.kernel_layout) { decode_generic(h, W_out); return; }
-    const int nkb = h.nkb, mask_rows = h.mask_rows, K_L = h.fmt.K_L;
+    const int CA = h.fmt.C_A, nkb = h.nkb / CA, mask_rows = h.mask_rows, K_L = h.fmt.K_L, K_B = K_L / CA;
     for (int64_t t = 0; t < h.n_items; ++t) {
         const int64_t rb = t / h.n_segs, sg = t % h.n_segs;
         const uint8_t* b = h.blob.data() + (size_t)h.item_off[t] * 16;
@@ -372,14 +396,16 @@ void decode_host(const HostMatrix& h, int8_t* W_out)
                 const uint8_t m = b[(size_t)(kb >> 2) * 128 + lane * 4 + (kb & 3)];
                 for (int j = 0; j < 8; ++j) {
                     if (!((m >> j) & 1)) continue;
-                    const uint8_t v = pay[(size_t)(pos >> 2) * 128 + lane * 4 + (pos & 3)];
+                    for (int ca = 0; ca < CA; ++ca) {
+                        const uint8_t v = pay[(size_t)(pos >> 2) * 128 * CA + 128 * ca + lane * 4 + (pos & 3)];
+                        const int64_t k = sg * K_L + (int64_t)ca * K_B + 32 * kb + 8 * tt + j;
+                        if (k >= h.K) continue;
+                        const int lo = (int)(v & 0xF) - 8;
+                        const int hi = (v >> 4) >= 8 ? (int)(v >> 4) - 16 : (int)(v >> 4);
+                        if (ra >= 0) W_out[(int64_t)ra * h.K + k] = (int8_t)lo;
+                        if (rbw >= 0) W_out[(int64_t)rbw * h.K + k] = (int8_t)hi;
+                    }
                     ++pos;
-                    const int64_t k = sg * K_L + 32 * kb + 8 * tt + j;
-                    if (k >= h.K) continue;
-                    const int lo = (int)(v & 0xF) - 8;
-                    const int hi = (v >> 4) >= 8 ? (int)(v >> 4) - 16 : (int)(v >> 4);
-                    if (ra >= 0) W_out[(int64_t)ra * h.K + k] = (int8_t)lo;
-                    if (rbw >= 0) W_out[(int64_t)rbw * h.K + k] = (int8_t)hi;
                 }
             }
         }

@@ -56,7 +56,9 @@ struct SpmmParams {
                                                 // segment count, n_strips * G
     int32_t s_local;            // local mode: strips a CTA may hold in shared memory (0 = direct mode)
     int32_t lut_rep;            // copies of the selector table in shared memory (8 or 32)
-    int32_t mask_rows, K_L;
+    int32_t mask_rows, K_L;     // mask words per lane and tile; tile width
+    int32_t fold_kb;            // C_A = 2: k-blocks per column area (a mask bit also covers the column that many
+                                // k-blocks further on); 0 for C_A = 1
     uint32_t slot_bytes;        // ring slot size (max tile blob + slack), multiple of 128
     int32_t x_fast;             // 2: K % 32 == 0 (16-byte loads); 1: K % 8 == 0 (4-byte loads); 0: bytes
     int32_t fp16_out;
@@ -414,15 +416,20 @@ __device__ __forceinline__ void store_rows(const StoreCtx p, const int (&v)[NT][
 // All addresses are 32-bit shared-memory addresses: slot_a = the staged tile, lut_a = selector
 // table + 4*lane, xb_a = this lane's first B-fragment of the tile's segment.
 // XP: X is staged packed (one word per lane, k-block and n-tile) instead of as int8 (two words).
-template <int NT, bool XP>
+// CA = column areas of the format: with CA = 2 one mask byte serves two k-blocks (kb and kb + fold_kb);
+// their payload bytes sit at the same position of two streams whose 128-byte rows alternate, so the
+// positions, the table entry and all address arithmetic are shared and only the window loads, the
+// shifts, the permutes and the MMA are done twice.
+template <int NT, bool XP, int CA>
 __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, uint32_t lut_stride,
                                              uint32_t xb_a, int xstride, int mask_rows, int lane,
-                                             int (&c)[NT][4])
+                                             int (&c)[NT][4], uint32_t x_fold)
 {
     const uint32_t mask_a = slot_a + 4u * lane;
     const uint32_t pay_a = slot_a + 128u * mask_rows + 4u * lane;
-    constexpr bool kPreX = NT <= 2;   // small N: fetch the X fragments together with the windows
+    constexpr bool kPreX = NT <= 2 && CA == 1;   // small N: fetch the X fragments together with the windows
     constexpr uint32_t kXStep = XP ? 16u : 32u;   // bytes of a token's row per k-block
+    constexpr int kRow = 128 * CA;                // bytes from one payload row of a stream to its next
     auto ldx = [&](uint32_t a) -> uint2 {         // the lane's two B-fragment words at address a
         if (XP) {
             const uint32_t q = lds32(a);
@@ -431,9 +438,12 @@ __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, ui
         return lds64(a);
     };
     uint32_t b8 = 0;                                     // 8 * (byte position in the lane's payload stream)
-    uint32_t cw0 = lds32_at<0>(pay_a), cw1 = lds32_at<128>(pay_a);   // carried window: the words at / after the position
+    uint32_t cw0[CA], cw1[CA];                           // carried window: the words at / after the position
+#pragma unroll
+    for (int ca = 0; ca < CA; ++ca) { cw0[ca] = lds32(pay_a + 128u * ca); cw1[ca] = lds32(pay_a + kRow + 128u * ca); }
+    const uint32_t xb_fold_a = xb_a + x_fold;            // X fragments of the second column area
     for (int w = 0; w < mask_rows; ++w) {
-        uint32_t pos[5], wm1[4], w0[4], w1[4], e[4];
+        uint32_t pos[5], wm1[CA][4], w0[CA][4], w1[CA][4], e[4];
         uint2 xf[4][kPreX ? NT : 1];
         const uint32_t mw = lds32(mask_a + 128u * w);
         pos[0] = b8;
@@ -446,10 +456,15 @@ __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, ui
         b8 = pos[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const uint32_t a = pay_a + ((pos[i + 1] >> 5) << 7);   // window at the block's END
-            wm1[i] = lds32_at<-128>(a);
-            w0[i] = lds32_at<0>(a);
-            w1[i] = lds32_at<128>(a);
+            const uint32_t a = pay_a + (pos[i + 1] >> 5) * (uint32_t)kRow;   // window at the block's END
+            wm1[0][i] = lds32_at<-kRow>(a);
+            w0[0][i] = lds32_at<0>(a);
+            w1[0][i] = lds32_at<kRow>(a);
+            if (CA == 2) {
+                wm1[CA - 1][i] = lds32_at<128 - kRow>(a);
+                w0[CA - 1][i] = lds32_at<128>(a);
+                w1[CA - 1][i] = lds32_at<128 + kRow>(a);
+            }
             e[i] = lds32(e[i]);
             if (kPreX) {
 #pragma unroll
@@ -458,21 +473,25 @@ __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, ui
         }
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            // first four bytes: the window starting at pos[i] (carried, or the previous block's)
-            const uint32_t s0 = (i == 0) ? cw0 : w0[i - 1];
-            const uint32_t s1 = (i == 0) ? cw1 : w1[i - 1];
-            const uint32_t lo = __funnelshift_r(s0, s1, pos[i]);
-            const uint32_t prev = __funnelshift_r(wm1[i], w0[i], pos[i + 1]);
-            const uint32_t d0 = prmt(lo, kFill, e[i]);
-            const uint32_t d1 = prmt(prev, kFill, e[i] >> 16);
-            const uint32_t e0 = d0 & 0x0F0F0F0Fu, e1 = d1 & 0x0F0F0F0Fu;
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt) {
-                const uint2 b = kPreX ? xf[i][nt] : ldx(xb_a + kXStep * (4 * w + i) + nt * 8 * xstride);
-                mma_s8(c[nt], d0, e0, d1, e1, b.x, b.y);
+            for (int ca = 0; ca < CA; ++ca) {
+                // first four bytes: the window starting at pos[i] (carried, or the previous block's)
+                const uint32_t s0 = (i == 0) ? cw0[ca] : w0[ca][i - 1];
+                const uint32_t s1 = (i == 0) ? cw1[ca] : w1[ca][i - 1];
+                const uint32_t lo = __funnelshift_r(s0, s1, pos[i]);
+                const uint32_t prev = __funnelshift_r(wm1[ca][i], w0[ca][i], pos[i + 1]);
+                const uint32_t d0 = prmt(lo, kFill, e[i]);
+                const uint32_t d1 = prmt(prev, kFill, e[i] >> 16);
+                const uint32_t e0 = d0 & 0x0F0F0F0Fu, e1 = d1 & 0x0F0F0F0Fu;
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const uint2 b = kPreX ? xf[i][nt] : ldx((ca ? xb_fold_a : xb_a) + kXStep * (4 * w + i) + nt * 8 * xstride);
+                    mma_s8(c[nt], d0, e0, d1, e1, b.x, b.y);
+                }
             }
         }
-        cw0 = w0[3]; cw1 = w1[3];
+#pragma unroll
+        for (int ca = 0; ca < CA; ++ca) { cw0[ca] = w0[ca][3]; cw1[ca] = w1[ca][3]; }
     }
 }
 
@@ -515,10 +534,11 @@ constexpr int kTimerWords = kWarpRec * kMaxWarpsPerCta * kMaxCtas;
 // kernel carries none of their clock reads and branches).
 // AM = chained call that leaves the per-token absmax of its fp16 output (separate too: the plain
 // fp16 store measured 2.5 % slower with the tracking compiled in behind a run-time flag).
-template <int NT, int STAGES, bool LA, bool TIMED, bool XP = false, bool AM = false>
+// CA = column areas of the weight format (2: folded tiles, N <= 8 only).
+template <int NT, int STAGES, bool LA, bool TIMED, bool XP = false, bool AM = false, int CA = 1>
 // (N <= 8 kernels are compiled for up to 20 warps: 80 registers instead of 90, which lets 12 instead of 10 warps of
 // two half-SM CTAs share an SM; more than 16 warps per full-SM CTA were measured and do not pay.)
-__global__ void __launch_bounds__(NT == 1 ? 640 : 512, 1) us_spmm_kernel(const SpmmParams p)
+__global__ void __launch_bounds__((NT == 1 && CA == 1) ? 640 : 512, 1) us_spmm_kernel(const SpmmParams p)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
@@ -915,7 +935,8 @@ __global__ void __launch_bounds__(NT == 1 ? 640 : 512, 1) us_spmm_kernel(const S
             const uint32_t slot_a = smem_u32(my_ring + (size_t)cur * p.slot_bytes);
             const uint32_t xb_a = XP ? smem_u32(x8) + (lane >> 2) * xstride + 4 * (lane & 3) + sgl * (p.K_L / 2)
                                      : smem_u32(x8) + (lane >> 2) * xstride + 8 * (lane & 3) + sgl * p.K_L;
-            process_tile<NT, XP>(slot_a, lut_a, 4u * (uint32_t)p.lut_rep, xb_a, xstride, p.mask_rows, lane, c);
+            process_tile<NT, XP, CA>(slot_a, lut_a, 4u * (uint32_t)p.lut_rep, xb_a, xstride, p.mask_rows, lane, c,
+                                     (uint32_t)p.fold_kb * (XP ? 16u : 32u));
             __syncwarp();
             const long long t2c = timing ? clock64() : 0;
 

@@ -145,6 +145,36 @@ def test_paper_layout_formats_round_trip_and_stats(b, fmt, M, K, s):
         b.us_destroy(h)
 
 
+# The folded kernel layout (two column areas: one mask bit covers rows i, i + 8 and columns j, j + K_L/2):
+# the library's own tile layout, the oracle's union rule and counts.
+@pytest.mark.parametrize("M,K,s,K_L", [(64, 1024, 0.5, 1024), (37, 300, 0.5, 256), (160, 2176, 0.7, 256),
+                                       (16, 256, 0.0, 256), (48, 512, 1.0, 512), (512, 2048, 0.6, 512)])
+@pytest.mark.parametrize("flags", [0, 2])
+def test_folded_kernel_layout_round_trip_and_stats(b, M, K, s, K_L, flags):
+    W = workloads.make_weight(M, K, s, seed=M + K + 7, row_varying=bool(flags & 2))
+    h = b.us_encode(W, fmt=(16, K_L, 2, 2), max_N=8, flags=b.US_ENCODE_HOST_ONLY | flags)
+    try:
+        assert (b.us_decode(h) == W).all()
+        st = b.us_get_stats(h)
+        assert st["fmt"] == (16, K_L, 2, 2)
+        order = b.us_get_row_order(h)
+        Wp = np.zeros((st["Mp"], K), np.int8)
+        Wp[order >= 0] = W[order[order >= 0]]
+        ref = oracle.encode(Wp, 16, K_L, 2, 2)["stats"]
+        for lib_key, ref_key in [("nnz", "nnz"), ("sum_P", "sum_P"), ("n_tiles", "n_lt"), ("Kp", "Kp"),
+                                 ("bytes_payload", "bytes_payload"), ("bytes_bitmap", "bytes_bitmap"),
+                                 ("bytes_offsets", "bytes_offsets")]:
+            assert st[lib_key] == ref[ref_key], lib_key
+        assert st["pmr"] == pytest.approx(ref["pmr"], rel=1e-12)
+        assert st["fill"] == pytest.approx(4 * ref["sum_P"] / (M * K), rel=1e-12)
+        assert st["bytes_payload_padded"] >= st["bytes_payload"] and st["bytes_payload_padded"] % 256 == 0
+    finally:
+        b.us_destroy(h)
+    with pytest.raises(b.UsError) as e:      # the pairing cost is defined for one column area
+        b.us_encode(W, fmt=(16, K_L, 2, 2), max_N=8, flags=b.US_ENCODE_HOST_ONLY | b.US_ENCODE_PAIR_ROWS)
+    assert e.value.status == 4
+
+
 def test_pack_int4(b):
     X = np.array([[1, -2, 7, -8, 0]], np.int8)
     assert list(b.pack_int4(X)[0]) == [0x1 | (0xE << 4), 0x7 | (0x8 << 4), 0x0]

@@ -353,3 +353,35 @@ def test_call_with_another_device_current_is_refused(b):
     finally:
         torch.cuda.set_device(0)
         sw.close()
+
+
+# ---- folded tiles: format (16, K_L, 2, 2), one mask bit per 2 x 2 weights (the paper's Q = 4 union), N <= 8 ----
+@pytest.mark.parametrize("M,K,s,K_L,flags", [
+    (1024, 1024, 0.5, 256, 0), (1024, 1024, 0.5, 512, 0), (1024, 1024, 0.5, 1024, 0),
+    (2000, 1000, 0.5, 512, 0),            # ragged rows and columns
+    (1030, 2056, 0.6, 1024, 2),           # ragged, rows sorted by density
+    (4096, 4096, 0.3, 512, 0), (4096, 4096, 0.7, 512, 0),
+    (512, 8192, 0.5, 2048, 0),            # long tiles
+    (4096, 11008, 0.5, 1024, 0),          # several K ranges
+    (16, 256, 0.0, 256, 0), (48, 512, 1.0, 512, 0),
+])
+def test_folded_format(b, M, K, s, K_L, flags):
+    seed = 600 + M % 91 + K % 83
+    W = workloads.make_weight(M, K, s, seed=seed, row_varying=bool(flags & 2))
+    X = workloads.make_x(K, 8, seed=seed)
+    s_w, s_x = workloads.make_scales(M, 8, seed=seed)
+    _check_case(b, W, X, [1, 3, 8], s_w, s_x, fmt=(16, K_L, 2, 2), flags=flags, max_N=8)
+
+
+def test_folded_format_70b_full_size(b):
+    """28672 x 8192 at 60 % sparsity in the folded format: every row, N = 8 and 1."""
+    W = workloads.make_weight(28672, 8192, 0.6, seed=500)
+    X = workloads.make_x(8192, 8, seed=500)
+    _check_case(b, W, X, [8, 1], fmt=(16, 1024, 2, 2), max_N=8)
+
+
+def test_folded_format_limits(b):
+    W = workloads.make_weight(256, 512, 0.5, seed=3)
+    with pytest.raises(b.UsError) as e:      # kernels for N <= 8 only
+        b.SparseWeight(W, None, fmt=(16, 256, 2, 2), max_N=16)
+    assert e.value.status == 4
