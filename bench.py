@@ -550,14 +550,14 @@ def sweep(binding, torch, workloads, l2, peak_gbs):
     # Bitmap-aware row pairing inside each strip (the per-strip form of Alg. 1): fewer union bits.
     run_case("attn7b_paired", 4096, 4096, 0.5, 201, [8], [True], flags=binding.US_ENCODE_PAIR_ROWS)
     run_case("ffn70b_up_paired", 28672, 8192, 0.6, 500, [8], [False], flags=binding.US_ENCODE_PAIR_ROWS)
-    # The paper's 2 x 2 union mask (Q = 4) in the folded kernel layout, N <= 8: more bytes, fewer decode
+    # The paper's 2 x 2 union mask (Q = 4) in the folded kernel layout: more bytes, fewer decode
     # instructions per weight. Same matrices and seeds as the rows above.
     for i, s in enumerate((0.3, 0.5, 0.7)):
-        run_case("attn7b_q4", 4096, 4096, s, 200 + i, [1, 8], [True], q4=True)
-    run_case("ffn7b_up_q4", 11008, 4096, 0.5, 300, [8], [True], row_varying=True, flags=SORT, q4=True)
-    run_case("ffn7b_down_q4", 4096, 11008, 0.5, 302, [8], [True], row_varying=True, flags=SORT, q4=True)
-    run_case("ffn70b_up_q4", 28672, 8192, 0.6, 500, [1, 8], [False], q4=True)
-    run_case("ffn70b_down_q4", 8192, 28672, 0.6, 501, [1, 8], [False], q4=True)
+        run_case("attn7b_q4", 4096, 4096, s, 200 + i, [1, 8, 16, 32], [True], q4=True)
+    run_case("ffn7b_up_q4", 11008, 4096, 0.5, 300, [8, 32], [True], row_varying=True, flags=SORT, q4=True)
+    run_case("ffn7b_down_q4", 4096, 11008, 0.5, 302, [8, 32], [True], row_varying=True, flags=SORT, q4=True)
+    run_case("ffn70b_up_q4", 28672, 8192, 0.6, 500, [1, 8, 16, 32, 64], [False], q4=True)
+    run_case("ffn70b_down_q4", 8192, 28672, 0.6, 501, [1, 8, 16, 32, 64], [False], q4=True)
     for s in (0.3, 0.5, 0.7):                                                                  # config 4
         rows.append(layer_chain(binding, torch, workloads, l2, s))
         rows.append(layer_chain_requant(binding, torch, workloads, l2, s))

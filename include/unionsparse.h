@@ -41,7 +41,7 @@ typedef enum us_status {
  * own array layout. The kernels implement H_L = 16, R_A = 2 with
  *   C_A = 1 (Q = 2): one bit covers rows i and i+8 of a 16-row strip; K_L a multiple of 128;
  *   C_A = 2 (Q = 4, the paper's 2 x 2 union): the bit also covers the column K_L/2 further on in the
- *            tile; K_L a multiple of 256; N <= 8 only (max_N <= 8), no chained calls, no row pairing;
+ *            tile; K_L a multiple of 256; no chained calls (us_spmm_requant with y_amax), no row pairing;
  * K_L up to 8192. Only such handles can be uploaded and multiplied. On a mask without structure
  * Q = 4 stores 1 - s^4 of the dense payload against 1 - s^2 for Q = 2 and is decoded with fewer
  * instructions per weight.

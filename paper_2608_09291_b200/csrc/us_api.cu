@@ -222,7 +222,7 @@ void plan_classes(us_handle* h, int n_cta, std::vector<uint32_t> (&sched)[4])
         // ranges become one); 5120 x 5120 12.0 -> 9.4 us (one range either way, but a CTA's share is
         // small and the staging pass and the freed shared memory count for more than the decode);
         // 13824 x 5120 15.7 -> 16.0 us (one range either way, long decode): not taken there.
-        if (nt <= 4 && h->host.fmt.C_A == 1) {   // (no packed-X kernel for folded tiles)
+        if (nt <= 4) {
             const int64_t n_segs = h->host.n_segs;
             const int64_t ranges = h->s_local[c] > 0 ? (n_segs + h->G[c] - 1) / h->G[c] : n_segs + 1;
             const bool small_share = nt >= 2 && (int64_t)h->host.blob.size() / std::max(1, n_cta) < 128 * 1024;
@@ -264,11 +264,16 @@ cudaError_t launch_st(const us::SpmmParams& p, bool xp, int grid, int block, int
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     const bool la = p.s_local > 0, timed = p.timers != nullptr;
-    if (p.fold_kb) {   // folded tiles (two column areas): N <= 8 kernels only, checked by the caller
-        if (la) return timed ? cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<1, ST, true, true, false, false, 2>, p)
-                             : cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<1, ST, true, false, false, false, 2>, p);
-        return timed ? cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<1, ST, false, true, false, false, 2>, p)
-                     : cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<1, ST, false, false, false, false, 2>, p);
+    if (p.fold_kb) {   // folded tiles (two column areas); stage timers for the N <= 8 kernels only
+        if (NT == 1 && timed)
+            return la ? cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<1, ST, true, true, false, false, 2>, p)
+                      : cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<1, ST, false, true, false, false, 2>, p);
+        if (NT <= 4 && xp && la) {
+            constexpr int NP = NT <= 4 ? NT : 4;
+            return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NP, ST, true, false, true, false, 2>, p);
+        }
+        return la ? cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, ST, true, false, false, false, 2>, p)
+                  : cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, ST, false, false, false, false, 2>, p);
     }
     if (p.y_amax) {   // chained call (never timed: enqueue_spmm leaves the timers off)
         if (NT <= 4 && xp && la) {
@@ -309,9 +314,11 @@ cudaError_t enable_large_smem_st(int bytes)
     if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, ST, false, false, false, true>, attr, bytes);
     constexpr int NP = NT <= 4 ? NT : 4;   // packed-X kernels exist for N <= 32
     if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NP, ST, true, false, true, true>, attr, bytes);
-    if (NT == 1) {   // folded tiles
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<1, ST, true, false, false, false, 2>, attr, bytes);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<1, ST, false, false, false, false, 2>, attr, bytes);
+    // folded tiles
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, ST, true, false, false, false, 2>, attr, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, ST, false, false, false, false, 2>, attr, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NP, ST, true, false, true, false, 2>, attr, bytes);
+    if (NT == 1) {
         if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<1, ST, true, true, false, false, 2>, attr, bytes);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<1, ST, false, true, false, false, 2>, attr, bytes);
     }
@@ -412,7 +419,8 @@ us_status enqueue_spmm(us_handle* h, const void* X, int32_t N, const void* x_sca
     p.X = static_cast<const uint8_t*>(X);
     p.x_scale = static_cast<const uint16_t*>(x_scale);
     p.Y = Y; p.acc = acc; p.cnt = cnt; p.err = h->d_err;
-    p.timers = (timers && !(chain && chain->y_amax)) ? h->d_timers : nullptr;
+    // (no stage-timer builds of the absmax-tracking kernels, nor of the folded-tile kernels for N > 8)
+    p.timers = (timers && !(chain && chain->y_amax) && !(hm.fmt.C_A == 2 && g.nt > 1)) ? h->d_timers : nullptr;
     p.M = (int32_t)hm.M; p.K = (int32_t)hm.K; p.N = N;
     p.n_strips = (int32_t)hm.n_strips; p.n_segs = (int32_t)hm.n_segs;
     p.mask_rows = hm.mask_rows; p.K_L = hm.fmt.K_L;
@@ -475,8 +483,6 @@ us_status us_encode(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_sca
         *out = h;
         return US_OK;
     }
-    // folded tiles (two column areas): kernels for N <= 8 only
-    if (hm.fmt.C_A == 2 && max_N > 8 && !host_only) { delete h; return US_ERR_UNSUPPORTED; }
     // the kernel's index arithmetic (exact division by multiplication) needs u * d < 2^40 for every
     // position u < n_items and divisor d <= n_items
     if (hm.n_items >= (1 << 20) || hm.n_segs >= (1 << 16)) {

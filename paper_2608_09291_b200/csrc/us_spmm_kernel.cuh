@@ -534,7 +534,7 @@ constexpr int kTimerWords = kWarpRec * kMaxWarpsPerCta * kMaxCtas;
 // kernel carries none of their clock reads and branches).
 // AM = chained call that leaves the per-token absmax of its fp16 output (separate too: the plain
 // fp16 store measured 2.5 % slower with the tracking compiled in behind a run-time flag).
-// CA = column areas of the weight format (2: folded tiles, N <= 8 only).
+// CA = column areas of the weight format (2: folded tiles).
 template <int NT, int STAGES, bool LA, bool TIMED, bool XP = false, bool AM = false, int CA = 1>
 // (N <= 8 kernels are compiled for up to 20 warps: 80 registers instead of 90, which lets 12 instead of 10 warps of
 // two half-SM CTAs share an SM; more than 16 warps per full-SM CTA were measured and do not pay.)

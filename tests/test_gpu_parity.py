@@ -380,8 +380,34 @@ def test_folded_format_70b_full_size(b):
     _check_case(b, W, X, [8, 1], fmt=(16, 1024, 2, 2), max_N=8)
 
 
+@pytest.mark.parametrize("M,K,s,K_L,Ns", [
+    (1024, 1024, 0.5, 512, [9, 16, 17, 32, 33, 64]),
+    (2000, 1000, 0.5, 256, [12, 24, 48]),
+    (5120, 5120, 0.5, 1024, [16, 32]),
+    (4096, 11008, 0.5, 1024, [16, 32, 64]),      # several K ranges / global split-K
+    (13824, 5120, 0.7, 1024, [16]),
+])
+def test_folded_format_wider_N(b, M, K, s, K_L, Ns):
+    seed = 650 + M % 91 + K % 83
+    W = workloads.make_weight(M, K, s, seed=seed)
+    X = workloads.make_x(K, max(Ns), seed=seed)
+    s_w, s_x = workloads.make_scales(M, max(Ns), seed=seed)
+    _check_case(b, W, X, Ns, s_w, s_x, fmt=(16, K_L, 2, 2), max_N=max(Ns))
+
+
 def test_folded_format_limits(b):
+    """Chained calls that leave an absmax have no folded-tile kernel: refused, not silently wrong."""
     W = workloads.make_weight(256, 512, 0.5, seed=3)
-    with pytest.raises(b.UsError) as e:      # kernels for N <= 8 only
-        b.SparseWeight(W, None, fmt=(16, 256, 2, 2), max_N=16)
-    assert e.value.status == 4
+    s_w, _ = workloads.make_scales(256, 8, seed=3)
+    sw = b.SparseWeight(W, s_w, fmt=(16, 256, 2, 2), max_N=8)
+    try:
+        X = torch.zeros((8, 512), dtype=torch.float16, device="cuda")
+        a, a2 = b.new_amax(), b.new_amax()
+        Y = torch.zeros((8, 256), dtype=torch.float16, device="cuda")
+        assert b._lib.us_spmm_requant(sw.handle, X.data_ptr(), 512, a.data_ptr(), 8, Y.data_ptr(), a2.data_ptr(), 0, 256, None) == 4
+        y = sw.spmm_requant(X, 8, b.absmax_f16(X))      # without an absmax output the plain kernels serve
+        torch.cuda.synchronize()
+        sw.check()
+        assert float(y.abs().max()) == 0.0
+    finally:
+        sw.close()
