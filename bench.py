@@ -62,13 +62,15 @@ def bytes_q1(stats: dict, N: int, fp16: bool) -> int:
     M, K = stats["M"], stats["K"]
     mp, kp = (M + 15) // 16 * 16, (K + 63) // 64 * 64
     n_lt = (mp // 16) * (kp // 64)
-    return (stats["nnz"] + 1) // 2 + mp * kp // 8 + 4 * (n_lt + 1) + io_bytes(M, K, N, fp16)
+    bits = stats.get("weight_bits", 4)
+    return (stats["nnz"] * bits + 7) // 8 + mp * kp // 8 + 4 * (n_lt + 1) + io_bytes(M, K, N, fp16)
 
 
 def bytes_dense_int4(stats: dict, N: int, fp16: bool) -> int:
-    """The same call on the dense INT4 weight (no bitmap, no pruning exploited)."""
+    """The same call on the dense weight at its own bit width (INT4, or INT2 for the W2A4 rows): no
+    bitmap, no pruning exploited."""
     M, K = stats["M"], stats["K"]
-    return (M * K + 1) // 2 + io_bytes(M, K, N, fp16)
+    return (M * K * stats.get("weight_bits", 4) + 7) // 8 + io_bytes(M, K, N, fp16)
 
 
 def measured_peaks():
@@ -498,10 +500,10 @@ TRAFFIC_BYTES_PER_LAUNCH_LARGE = 102_112_256  # 28672x8192, s = 0.6, N = 8, int3
 def sweep(binding, torch, workloads, l2, peak_gbs):
     rows = []
 
-    def run_case(name, M, K, s, seed, Ns, outs, row_varying=False, flags=0, q4=False):
+    def run_case(name, M, K, s, seed, Ns, outs, row_varying=False, flags=0, q4=False, w2=False):
         """q4: the folded format (16, K_L, 2, 2) -- one mask bit per 2 x 2 weights -- at the K_L the
         library picks for this shape, instead of the default (16, K_L, 2, 1)."""
-        W = workloads.make_weight(M, K, s, seed, row_varying)
+        W = workloads.make_weight_w2(M, K, s, seed) if w2 else workloads.make_weight(M, K, s, seed, row_varying)
         Nmax = max(Ns)
         X = workloads.make_x(K, Nmax, seed)
         s_w, s_x = workloads.make_scales(M, Nmax, seed)
@@ -509,8 +511,10 @@ def sweep(binding, torch, workloads, l2, peak_gbs):
         st = binding.us_get_stats(probe)
         binding.us_destroy(probe)
         fmt = None
-        if q4:
+        if q4 or w2:   # w2: INT2 weights, which live in the folded format only
             fmt = (16, st["fmt"][1], 2, 2)
+            if w2:
+                flags |= binding.US_ENCODE_W2
             probe = binding.us_encode(W, None, fmt, Nmax, binding.US_ENCODE_HOST_ONLY | flags)
             st = binding.us_get_stats(probe)
             binding.us_destroy(probe)
@@ -532,6 +536,7 @@ def sweep(binding, torch, workloads, l2, peak_gbs):
                              "bytes_dense_int4": dn, "us_dense_int4_at_8tbs": dn / CONTRACT_PEAK_GBS / 1e3,
                              "dense_equiv_tops": 2.0 * M * K * N / t / 1e12, "replicas": R,
                              "pmr": case.stats["pmr"], "format": list(case.stats["fmt"]),
+                             "weight_bits": case.stats["weight_bits"],
                              "kernel": kernel_label(binding, case.sw[0].handle, N)})
         case.close()
         del case
@@ -558,6 +563,10 @@ def sweep(binding, torch, workloads, l2, peak_gbs):
     run_case("ffn7b_down_q4", 4096, 11008, 0.5, 302, [8, 32], [True], row_varying=True, flags=SORT, q4=True)
     run_case("ffn70b_up_q4", 28672, 8192, 0.6, 500, [1, 8, 16, 32, 64], [False], q4=True)
     run_case("ffn70b_down_q4", 8192, 28672, 0.6, 501, [1, 8, 16, 32, 64], [False], q4=True)
+    # W2A4 (Sec. VII-B): INT2 weights, one payload byte per union-mask bit of the folded format
+    run_case("attn7b_w2a4", 4096, 4096, 0.5, 201, [1, 8, 32], [True], w2=True)
+    run_case("ffn70b_up_w2a4", 28672, 8192, 0.6, 500, [1, 8, 16, 32], [False], w2=True)
+    run_case("ffn70b_down_w2a4", 8192, 28672, 0.6, 501, [1, 8, 16, 32], [False], w2=True)
     for s in (0.3, 0.5, 0.7):                                                                  # config 4
         rows.append(layer_chain(binding, torch, workloads, l2, s))
         rows.append(layer_chain_requant(binding, torch, workloads, l2, s))

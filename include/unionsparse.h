@@ -57,15 +57,17 @@ typedef struct us_stats {
     int64_t nnz;                  /* true nonzeros                                          */
     int64_t n_tiles;              /* local tiles (one offset each)                          */
     int64_t sum_P;                /* sum over tiles of P_t = active union-mask bits         */
-    int64_t bytes_payload;        /* ceil(Q * sum_P / 2): the packed INT4 values            */
+    int64_t bytes_payload;        /* ceil(Q * sum_P * weight_bits / 8): the packed values   */
     int64_t bytes_payload_padded; /* payload bytes as stored (kernel layout: lane streams padded
                                      per tile; the paper's layout stores no padding)        */
     int64_t bytes_bitmap;         /* union bitmaps                                          */
     int64_t bytes_offsets;        /* 4 * (n_tiles + 1)                                      */
     int64_t bytes_total;          /* bytes_payload_padded + bytes_bitmap + bytes_offsets    */
-    double  pmr;                  /* Eq. 1: 0.5 * nnz / (bytes_bitmap + bytes_offsets)      */
+    double  pmr;                  /* Eq. 1: B_w * nnz / (bytes_bitmap + bytes_offsets), B_w = weight_bits / 8 */
     double  fill;                 /* stored values / (M*K) = Q * sum_P / (M*K)              */
     us_format fmt;                /* the format in use                                      */
+    int32_t weight_bits;          /* 4, or 2 for a US_ENCODE_W2 handle                      */
+    int32_t reserved;
 } us_stats;
 
 typedef struct us_handle us_handle;
@@ -77,6 +79,12 @@ typedef struct us_handle us_handle;
                                   so that rows of similar density share a strip; the output
                                   row order of us_spmm is unchanged (folded into the store)  */
 
+#define US_ENCODE_W2 8u        /* W2A4 (paper Sec. VII-B, the W2A4 kernel figure): the weights are INT2, values in
+                                  [-2, 1] (others: US_ERR_VALUE_RANGE). Needs the format (16, K_L, 2, 2): the
+                                  four 2-bit values under one union-mask bit fill exactly one payload byte
+                                  (bits 1:0 = W[i][k] + 2, 3:2 = W[i+8][k] + 2, 5:4 and 7:6 the same at column
+                                  k + K_L/2), so the decode stays byte-granular. Other formats:
+                                  US_ERR_UNSUPPORTED. No chained calls, no row pairing.                  */
 #define US_ENCODE_PAIR_ROWS 4u /* bitmap-aware row reordering (paper Sec. V-B, Alg. 1) in its
                                   per-strip form: inside every 16-row strip (after SORT_ROWS, if
                                   also given) choose which two rows share each union-mask row so

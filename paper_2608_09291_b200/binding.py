@@ -21,6 +21,7 @@ US_OK = 0
 US_ENCODE_HOST_ONLY = 1
 US_ENCODE_SORT_ROWS = 2
 US_ENCODE_PAIR_ROWS = 4
+US_ENCODE_W2 = 8
 
 EXPORTS = ["us_encode", "us_get_stats", "us_decode", "us_get_row_order", "us_spmm", "us_spmm_static_scratch",
            "us_spmm_requant", "us_absmax_f16", "us_quantize_f16",
@@ -36,7 +37,8 @@ class us_stats(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int64) for n in (
         "M", "K", "Mp", "Kp", "nnz", "n_tiles", "sum_P", "bytes_payload", "bytes_payload_padded",
         "bytes_bitmap", "bytes_offsets", "bytes_total")] + [
-        ("pmr", ctypes.c_double), ("fill", ctypes.c_double), ("fmt", us_format)]
+        ("pmr", ctypes.c_double), ("fill", ctypes.c_double), ("fmt", us_format),
+        ("weight_bits", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
 _vp = ctypes.c_void_p

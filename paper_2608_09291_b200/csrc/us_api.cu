@@ -82,7 +82,8 @@ struct LaunchGeom {
 // stream's end (rows are 128 bytes per column area).
 uint32_t slot_bytes_for(const us::HostMatrix& hm)
 {
-    return (hm.max_item_bytes + 256u * (uint32_t)hm.fmt.C_A + 127u) & ~127u;
+    const uint32_t streams = hm.w2 ? 1u : (uint32_t)hm.fmt.C_A;
+    return (hm.max_item_bytes + 256u * streams + 127u) & ~127u;
 }
 
 int64_t x_bytes(int nt, int64_t G, int K_L, bool xp)
@@ -222,7 +223,7 @@ void plan_classes(us_handle* h, int n_cta, std::vector<uint32_t> (&sched)[4])
         // ranges become one); 5120 x 5120 12.0 -> 9.4 us (one range either way, but a CTA's share is
         // small and the staging pass and the freed shared memory count for more than the decode);
         // 13824 x 5120 15.7 -> 16.0 us (one range either way, long decode): not taken there.
-        if (nt <= 4) {
+        if (nt <= 4 && !h->host.w2) {   // (no packed-X kernel for INT2 weights)
             const int64_t n_segs = h->host.n_segs;
             const int64_t ranges = h->s_local[c] > 0 ? (n_segs + h->G[c] - 1) / h->G[c] : n_segs + 1;
             const bool small_share = nt >= 2 && (int64_t)h->host.blob.size() / std::max(1, n_cta) < 128 * 1024;
@@ -264,6 +265,9 @@ cudaError_t launch_st(const us::SpmmParams& p, bool xp, int grid, int block, int
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     const bool la = p.s_local > 0, timed = p.timers != nullptr;
+    if (p.w2)   // INT2 weights in folded tiles: plain kernels only (no packed X, timers or absmax)
+        return la ? cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, ST, true, false, false, false, 2, true>, p)
+                  : cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, ST, false, false, false, false, 2, true>, p);
     if (p.fold_kb) {   // folded tiles (two column areas); stage timers for the N <= 8 kernels only
         if (NT == 1 && timed)
             return la ? cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<1, ST, true, true, false, false, 2>, p)
@@ -314,7 +318,9 @@ cudaError_t enable_large_smem_st(int bytes)
     if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, ST, false, false, false, true>, attr, bytes);
     constexpr int NP = NT <= 4 ? NT : 4;   // packed-X kernels exist for N <= 32
     if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NP, ST, true, false, true, true>, attr, bytes);
-    // folded tiles
+    // folded tiles, INT4 and INT2
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, ST, true, false, false, false, 2, true>, attr, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, ST, false, false, false, false, 2, true>, attr, bytes);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, ST, true, false, false, false, 2>, attr, bytes);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, ST, false, false, false, false, 2>, attr, bytes);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NP, ST, true, false, true, false, 2>, attr, bytes);
@@ -420,11 +426,12 @@ us_status enqueue_spmm(us_handle* h, const void* X, int32_t N, const void* x_sca
     p.x_scale = static_cast<const uint16_t*>(x_scale);
     p.Y = Y; p.acc = acc; p.cnt = cnt; p.err = h->d_err;
     // (no stage-timer builds of the absmax-tracking kernels, nor of the folded-tile kernels for N > 8)
-    p.timers = (timers && !(chain && chain->y_amax) && !(hm.fmt.C_A == 2 && g.nt > 1)) ? h->d_timers : nullptr;
+    p.timers = (timers && !(chain && chain->y_amax) && !(hm.fmt.C_A == 2 && g.nt > 1) && !hm.w2) ? h->d_timers : nullptr;
     p.M = (int32_t)hm.M; p.K = (int32_t)hm.K; p.N = N;
     p.n_strips = (int32_t)hm.n_strips; p.n_segs = (int32_t)hm.n_segs;
     p.mask_rows = hm.mask_rows; p.K_L = hm.fmt.K_L;
     p.fold_kb = hm.fmt.C_A == 2 ? hm.nkb / 2 : 0;
+    p.w2 = hm.w2 ? 1 : 0;
     p.slot_bytes = g.slot_bytes;
     p.x_fast = (hm.K % 32 == 0) ? 2 : (hm.K % 8 == 0) ? 1 : 0;
     p.fp16_out = x_scale ? 1 : 0;

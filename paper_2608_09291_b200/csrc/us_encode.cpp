@@ -236,6 +236,10 @@ us_status encode_host(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_s
     h.M = M; h.K = K; h.fmt = fmt;
     h.kernel_layout = fmt.H_L == 16 && fmt.R_A == 2 && fmt.K_L <= 8192 &&
                       ((fmt.C_A == 1 && fmt.K_L % 128 == 0) || (fmt.C_A == 2 && fmt.K_L % 256 == 0));
+    h.w2 = (flags & US_ENCODE_W2) != 0;
+    // INT2 weights: only in the folded kernel layout, where a mask bit's four values fill one byte
+    if (h.w2 && !(h.kernel_layout && fmt.C_A == 2)) { h = HostMatrix(); return US_ERR_UNSUPPORTED; }
+    if (h.w2 && (flags & US_ENCODE_PAIR_ROWS)) { h = HostMatrix(); return US_ERR_UNSUPPORTED; }
     if (!h.kernel_layout) {
         // a valid IE-BME format without a kernel: the paper's arrays, for statistics and decoding
         if (!(flags & US_ENCODE_HOST_ONLY)) return US_ERR_UNSUPPORTED;
@@ -280,6 +284,9 @@ us_status encode_host(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_s
 
     // ---- build every tile blob (parallel over strips) ------------------------------------
     const int K_L = fmt.K_L, CA = fmt.C_A, nkb = h.nkb / CA, mask_rows = h.mask_rows;   // nkb: mask bytes per lane
+    const bool w2 = h.w2;
+    const int vmin = w2 ? -2 : -8, vmax = w2 ? 1 : 7;
+    const int SR = w2 ? 1 : CA;   // payload streams per lane (INT2: the two column areas share a byte)
     const int K_B = K_L / CA;                                                            // columns per column area
     const int64_t mask_bytes = (int64_t)mask_rows * 128;
     std::vector<std::vector<uint8_t>> blobs(h.n_items);
@@ -318,15 +325,19 @@ us_status encode_host(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_s
                     if (!any) continue;
                     bool range_ok = true;
                     for (int ca = 0; ca < CA; ++ca)
-                        for (int r = 0; r < 2; ++r) range_ok = range_ok && v[ca][r] >= -8 && v[ca][r] <= 7;
+                        for (int r = 0; r < 2; ++r) range_ok = range_ok && v[ca][r] >= vmin && v[ca][r] <= vmax;
                     if (!range_ok) { bad.store(1); continue; }
                     for (int ca = 0; ca < CA; ++ca) my_nnz += (v[ca][0] != 0) + (v[ca][1] != 0);
                     const int kb = kk >> 5, t = (kk >> 3) & 3, j = kk & 7;
                     const int lane = 4 * g + t;
                     mask[(size_t)lane * nkb + kb] |= (uint8_t)(1u << j);
                     const size_t at = (size_t)lane * nkb * 8 + len[lane]++;
-                    stream[at] = (uint8_t)(((v[0][1] & 0xF) << 4) | ((v[0][0] + 8) & 0xF));
-                    if (CA == 2) stream2[at] = (uint8_t)(((v[1][1] & 0xF) << 4) | ((v[1][0] + 8) & 0xF));
+                    if (w2) {
+                        stream[at] = (uint8_t)((v[0][0] + 2) | ((v[0][1] + 2) << 2) | ((v[1][0] + 2) << 4) | ((v[1][1] + 2) << 6));
+                    } else {
+                        stream[at] = (uint8_t)(((v[0][1] & 0xF) << 4) | ((v[0][0] + 8) & 0xF));
+                        if (CA == 2) stream2[at] = (uint8_t)(((v[1][1] & 0xF) << 4) | ((v[1][0] + 8) & 0xF));
+                    }
                 }
             }
             int maxlen = 0;
@@ -334,14 +345,14 @@ us_status encode_host(const int8_t* W, int64_t M, int64_t K, const uint16_t* w_s
             const int J = (maxlen + 3) / 4;
             std::vector<uint8_t>& b = blobs[rb * h.n_segs + sg];
             // payload rows of 32 lane words; with C_A = 2 the rows of the two streams alternate
-            b.assign((size_t)mask_bytes + (size_t)J * 128 * CA, 0);
+            b.assign((size_t)mask_bytes + (size_t)J * 128 * SR, 0);
             for (int l = 0; l < 32; ++l) {
                 for (int w = 0; w < mask_rows; ++w)
                     std::memcpy(&b[(size_t)w * 128 + l * 4], &mask[(size_t)l * nkb + 4 * w], 4);
                 const uint8_t* s = &stream[(size_t)l * nkb * 8];
                 for (int i = 0; i < len[l]; ++i)
-                    b[(size_t)mask_bytes + (size_t)(i >> 2) * 128 * CA + l * 4 + (i & 3)] = s[i];
-                if (CA == 2) {
+                    b[(size_t)mask_bytes + (size_t)(i >> 2) * 128 * SR + l * 4 + (i & 3)] = s[i];
+                if (SR == 2) {
                     const uint8_t* s2 = &stream2[(size_t)l * nkb * 8];
                     for (int i = 0; i < len[l]; ++i)
                         b[(size_t)mask_bytes + (size_t)(i >> 2) * 256 + 128 + l * 4 + (i & 3)] = s2[i];
@@ -397,11 +408,18 @@ void decode_host(const HostMatrix& h, int8_t* W_out)
                 for (int j = 0; j < 8; ++j) {
                     if (!((m >> j) & 1)) continue;
                     for (int ca = 0; ca < CA; ++ca) {
-                        const uint8_t v = pay[(size_t)(pos >> 2) * 128 * CA + 128 * ca + lane * 4 + (pos & 3)];
                         const int64_t k = sg * K_L + (int64_t)ca * K_B + 32 * kb + 8 * tt + j;
                         if (k >= h.K) continue;
-                        const int lo = (int)(v & 0xF) - 8;
-                        const int hi = (v >> 4) >= 8 ? (int)(v >> 4) - 16 : (int)(v >> 4);
+                        int lo, hi;
+                        if (h.w2) {
+                            const uint8_t v = pay[(size_t)(pos >> 2) * 128 + lane * 4 + (pos & 3)];
+                            lo = (int)((v >> (4 * ca)) & 3) - 2;
+                            hi = (int)((v >> (4 * ca + 2)) & 3) - 2;
+                        } else {
+                            const uint8_t v = pay[(size_t)(pos >> 2) * 128 * CA + 128 * ca + lane * 4 + (pos & 3)];
+                            lo = (int)(v & 0xF) - 8;
+                            hi = (v >> 4) >= 8 ? (int)(v >> 4) - 16 : (int)(v >> 4);
+                        }
                         if (ra >= 0) W_out[(int64_t)ra * h.K + k] = (int8_t)lo;
                         if (rbw >= 0) W_out[(int64_t)rbw * h.K + k] = (int8_t)hi;
                     }
@@ -418,7 +436,10 @@ void fill_stats(const HostMatrix& h, us_stats* st)
     st->M = h.M; st->K = h.K; st->Mp = h.Mp; st->Kp = h.Kp;
     st->nnz = h.nnz;
     st->sum_P = h.sum_P;
-    st->bytes_payload = ((int64_t)Q * h.sum_P + 1) / 2;
+    const int bits = h.w2 ? 2 : 4;
+    st->bytes_payload = ((int64_t)Q * h.sum_P * bits + 7) / 8;
+    st->weight_bits = bits;
+    st->reserved = 0;
     if (h.kernel_layout) {
         st->n_tiles = h.n_items;
         st->bytes_payload_padded = h.bytes_payload_padded;
@@ -431,7 +452,7 @@ void fill_stats(const HostMatrix& h, us_stats* st)
         st->bytes_offsets = 4 * (h.gen.n_lt + 1);
     }
     st->bytes_total = st->bytes_payload_padded + st->bytes_bitmap + st->bytes_offsets;
-    st->pmr = 0.5 * (double)h.nnz / (double)(st->bytes_bitmap + st->bytes_offsets);
+    st->pmr = (bits / 8.0) * (double)h.nnz / (double)(st->bytes_bitmap + st->bytes_offsets);
     st->fill = (double)Q * (double)h.sum_P / ((double)h.M * (double)h.K);
     st->fmt = h.fmt;
 }

@@ -40,6 +40,7 @@ struct HostMatrix {
     int64_t M = 0, K = 0, Mp = 0, Kp = 0;
     us_format fmt{16, 1024, 2, 1};
     bool kernel_layout = true;   // false: generic arrays only (host-only formats)
+    bool w2 = false;             // INT2 weights: one payload byte per union-mask bit of the (16, K_L, 2, 2) format
     GenericArrays gen;
     int32_t nkb = 0;        // k-blocks (32 columns) per tile
     int32_t mask_rows = 0;  // nkb / 4

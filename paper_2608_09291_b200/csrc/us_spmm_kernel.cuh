@@ -57,6 +57,7 @@ struct SpmmParams {
     int32_t s_local;            // local mode: strips a CTA may hold in shared memory (0 = direct mode)
     int32_t lut_rep;            // copies of the selector table in shared memory (8 or 32)
     int32_t mask_rows, K_L;     // mask words per lane and tile; tile width
+    int32_t w2;                 // INT2 weights (the W2 kernel instantiations)
     int32_t fold_kb;            // C_A = 2: k-blocks per column area (a mask bit also covers the column that many
                                 // k-blocks further on); 0 for C_A = 1
     uint32_t slot_bytes;        // ring slot size (max tile blob + slack), multiple of 128
@@ -77,7 +78,8 @@ constexpr int kLutRepMax = 32;   // copies of the selector table: lane l reads c
                              // cost ~0.4 extra wavefronts per lookup (lanes sharing a copy collide only
                              // when their entries fall in the same bank) and free 24 KB for more warps.
 constexpr uint32_t kLutScratchBytes = 256 * 4;   // one unreplicated copy, built first
-constexpr uint32_t kFill = 0x08080808u;
+constexpr uint32_t kFill = 0x08080808u;      // INT4 payload byte of a cleared mask bit: w_hi = 0, w_lo + 8 = 8
+constexpr uint32_t kFillW2 = 0xAAAAAAAAu;    // INT2 payload byte of a cleared mask bit: four fields of 0 + 2
 constexpr uint32_t kErrTimeout = 1;
 constexpr int kNoRow = -2;        // "row ids not loaded yet" marker (-1 is a padding row)
 constexpr int kClaimWords = 96;   // shared-memory words of the claim counter and its neighbours
@@ -420,7 +422,11 @@ __device__ __forceinline__ void store_rows(const StoreCtx p, const int (&v)[NT][
 // their payload bytes sit at the same position of two streams whose 128-byte rows alternate, so the
 // positions, the table entry and all address arithmetic are shared and only the window loads, the
 // shifts, the permutes and the MMA are done twice.
-template <int NT, bool XP, int CA>
+// W2 (with CA = 2): INT2 weights. The byte of a set mask bit holds the bit's four 2-bit values (each + 2): low
+// nibble = column area 0 (bits 1:0 row g, 3:2 row g + 8), high nibble = column area 1. One stream, gathered as
+// for CA = 1, then split: fragment rows g take the nibble 4 * (w_hi + 2) + (w_lo + 2), rows g + 8 its low two
+// bits w_lo + 2; with S = sum of x over the tile's columns, Y_lo = E - 2 S and Y_hi = (RAW - E) / 4 - 2 S.
+template <int NT, bool XP, int CA, bool W2 = false>
 __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, uint32_t lut_stride,
                                              uint32_t xb_a, int xstride, int mask_rows, int lane,
                                              int (&c)[NT][4], uint32_t x_fold)
@@ -429,7 +435,8 @@ __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, ui
     const uint32_t pay_a = slot_a + 128u * mask_rows + 4u * lane;
     constexpr bool kPreX = NT <= 2 && CA == 1;   // small N: fetch the X fragments together with the windows
     constexpr uint32_t kXStep = XP ? 16u : 32u;   // bytes of a token's row per k-block
-    constexpr int kRow = 128 * CA;                // bytes from one payload row of a stream to its next
+    constexpr int SR = W2 ? 1 : CA;               // payload streams per lane
+    constexpr int kRow = 128 * SR;                // bytes from one payload row of a stream to its next
     auto ldx = [&](uint32_t a) -> uint2 {         // the lane's two B-fragment words at address a
         if (XP) {
             const uint32_t q = lds32(a);
@@ -438,12 +445,12 @@ __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, ui
         return lds64(a);
     };
     uint32_t b8 = 0;                                     // 8 * (byte position in the lane's payload stream)
-    uint32_t cw0[CA], cw1[CA];                           // carried window: the words at / after the position
+    uint32_t cw0[SR], cw1[SR];                           // carried window: the words at / after the position
 #pragma unroll
-    for (int ca = 0; ca < CA; ++ca) { cw0[ca] = lds32(pay_a + 128u * ca); cw1[ca] = lds32(pay_a + kRow + 128u * ca); }
+    for (int ca = 0; ca < SR; ++ca) { cw0[ca] = lds32(pay_a + 128u * ca); cw1[ca] = lds32(pay_a + kRow + 128u * ca); }
     const uint32_t xb_fold_a = xb_a + x_fold;            // X fragments of the second column area
     for (int w = 0; w < mask_rows; ++w) {
-        uint32_t pos[5], wm1[CA][4], w0[CA][4], w1[CA][4], e[4];
+        uint32_t pos[5], wm1[SR][4], w0[SR][4], w1[SR][4], e[4];
         uint2 xf[4][kPreX ? NT : 1];
         const uint32_t mw = lds32(mask_a + 128u * w);
         pos[0] = b8;
@@ -460,10 +467,10 @@ __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, ui
             wm1[0][i] = lds32_at<-kRow>(a);
             w0[0][i] = lds32_at<0>(a);
             w1[0][i] = lds32_at<kRow>(a);
-            if (CA == 2) {
-                wm1[CA - 1][i] = lds32_at<128 - kRow>(a);
-                w0[CA - 1][i] = lds32_at<128>(a);
-                w1[CA - 1][i] = lds32_at<128 + kRow>(a);
+            if (SR == 2) {
+                wm1[SR - 1][i] = lds32_at<128 - kRow>(a);
+                w0[SR - 1][i] = lds32_at<128>(a);
+                w1[SR - 1][i] = lds32_at<128 + kRow>(a);
             }
             e[i] = lds32(e[i]);
             if (kPreX) {
@@ -473,6 +480,24 @@ __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, ui
         }
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
+            if (W2) {
+                const uint32_t s0 = (i == 0) ? cw0[0] : w0[0][i - 1];
+                const uint32_t s1 = (i == 0) ? cw1[0] : w1[0][i - 1];
+                const uint32_t lo = __funnelshift_r(s0, s1, pos[i]);
+                const uint32_t prev = __funnelshift_r(wm1[0][i], w0[0][i], pos[i + 1]);
+                const uint32_t g0 = prmt(lo, kFillW2, e[i]);
+                const uint32_t g1 = prmt(prev, kFillW2, e[i] >> 16);
+#pragma unroll
+                for (int ca = 0; ca < 2; ++ca) {
+                    const uint32_t d0 = (ca ? g0 >> 4 : g0) & 0x0F0F0F0Fu, d1 = (ca ? g1 >> 4 : g1) & 0x0F0F0F0Fu;
+                    const uint32_t e0 = d0 & 0x03030303u, e1 = d1 & 0x03030303u;
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        const uint2 b = ldx((ca ? xb_fold_a : xb_a) + kXStep * (4 * w + i) + nt * 8 * xstride);
+                        mma_s8(c[nt], d0, e0, d1, e1, b.x, b.y);
+                    }
+                }
+            } else {
 #pragma unroll
             for (int ca = 0; ca < CA; ++ca) {
                 // first four bytes: the window starting at pos[i] (carried, or the previous block's)
@@ -489,9 +514,10 @@ __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, ui
                     mma_s8(c[nt], d0, e0, d1, e1, b.x, b.y);
                 }
             }
+            }
         }
 #pragma unroll
-        for (int ca = 0; ca < CA; ++ca) { cw0[ca] = w0[ca][3]; cw1[ca] = w1[ca][3]; }
+        for (int ca = 0; ca < SR; ++ca) { cw0[ca] = w0[ca][3]; cw1[ca] = w1[ca][3]; }
     }
 }
 
@@ -535,7 +561,8 @@ constexpr int kTimerWords = kWarpRec * kMaxWarpsPerCta * kMaxCtas;
 // AM = chained call that leaves the per-token absmax of its fp16 output (separate too: the plain
 // fp16 store measured 2.5 % slower with the tracking compiled in behind a run-time flag).
 // CA = column areas of the weight format (2: folded tiles).
-template <int NT, int STAGES, bool LA, bool TIMED, bool XP = false, bool AM = false, int CA = 1>
+// W2 = INT2 weights (folded format only).
+template <int NT, int STAGES, bool LA, bool TIMED, bool XP = false, bool AM = false, int CA = 1, bool W2 = false>
 // (N <= 8 kernels are compiled for up to 20 warps: 80 registers instead of 90, which lets 12 instead of 10 warps of
 // two half-SM CTAs share an SM; more than 16 warps per full-SM CTA were measured and do not pay.)
 __global__ void __launch_bounds__((NT == 1 && CA == 1) ? 640 : 512, 1) us_spmm_kernel(const SpmmParams p)
@@ -935,7 +962,7 @@ __global__ void __launch_bounds__((NT == 1 && CA == 1) ? 640 : 512, 1) us_spmm_k
             const uint32_t slot_a = smem_u32(my_ring + (size_t)cur * p.slot_bytes);
             const uint32_t xb_a = XP ? smem_u32(x8) + (lane >> 2) * xstride + 4 * (lane & 3) + sgl * (p.K_L / 2)
                                      : smem_u32(x8) + (lane >> 2) * xstride + 8 * (lane & 3) + sgl * p.K_L;
-            process_tile<NT, XP, CA>(slot_a, lut_a, 4u * (uint32_t)p.lut_rep, xb_a, xstride, p.mask_rows, lane, c,
+            process_tile<NT, XP, CA, W2>(slot_a, lut_a, 4u * (uint32_t)p.lut_rep, xb_a, xstride, p.mask_rows, lane, c,
                                      (uint32_t)p.fold_kb * (XP ? 16u : 32u));
             __syncwarp();
             const long long t2c = timing ? clock64() : 0;
@@ -955,10 +982,17 @@ __global__ void __launch_bounds__((NT == 1 && CA == 1) ? 640 : 512, 1) us_spmm_k
             for (int nt = 0; nt < NT; ++nt) {
                 const int n0 = nt * 8 + t2;
                 const int s0 = sxp[n0] >> 4, s1 = sxp[n0 + 1] >> 4;
-                y[nt][0] += (c[nt][2] >> 4) - 8 * s0;                 // strip row g
-                y[nt][1] += (c[nt][3] >> 4) - 8 * s1;
-                y[nt][2] += (c[nt][0] - c[nt][2]) >> 8;               // strip row g + 8
-                y[nt][3] += (c[nt][1] - c[nt][3]) >> 8;
+                if (W2) {
+                    y[nt][0] += (c[nt][2] >> 4) - 2 * s0;                  // strip row g
+                    y[nt][1] += (c[nt][3] >> 4) - 2 * s1;
+                    y[nt][2] += ((c[nt][0] - c[nt][2]) >> 6) - 2 * s0;     // strip row g + 8
+                    y[nt][3] += ((c[nt][1] - c[nt][3]) >> 6) - 2 * s1;
+                } else {
+                    y[nt][0] += (c[nt][2] >> 4) - 8 * s0;                 // strip row g
+                    y[nt][1] += (c[nt][3] >> 4) - 8 * s1;
+                    y[nt][2] += (c[nt][0] - c[nt][2]) >> 8;               // strip row g + 8
+                    y[nt][3] += (c[nt][1] - c[nt][3]) >> 8;
+                }
             }
             ++y_n;
             // the run goes on if this warp's next tile is the next segment of the same strip

@@ -32,6 +32,19 @@ def make_weight(M: int, K: int, sparsity: float, seed: int, row_varying: bool = 
     return W
 
 
+def make_weight_w2(M: int, K: int, sparsity: float, seed: int) -> np.ndarray:
+    """INT2 weights for the W2A4 rows: the mask of make_weight(seed), kept values uniform on
+    {-2, -1, 1} (the nonzero values of [-2, 1])."""
+    W4 = make_weight(M, K, sparsity, seed)
+    out = np.zeros_like(W4)
+    for c, r0 in enumerate(range(0, M, ROW_CHUNK)):
+        rows = min(ROW_CHUNK, M - r0)
+        rng = np.random.default_rng([seed, c, 2])
+        v = np.array([-2, -1, 1], dtype=np.int8)[rng.integers(0, 3, (rows, K))]
+        out[r0:r0 + rows] = np.where(W4[r0:r0 + rows] != 0, v, 0)
+    return out
+
+
 def make_x(K: int, N_max: int, seed: int) -> np.ndarray:
     """Activations, int8 values uniform on [-8,7], token-major (N_max, K)."""
     rng = np.random.default_rng([seed, _X_STREAM])

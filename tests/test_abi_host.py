@@ -175,6 +175,44 @@ def test_folded_kernel_layout_round_trip_and_stats(b, M, K, s, K_L, flags):
     assert e.value.status == 4
 
 
+# W2A4: INT2 weights in the folded layout, one payload byte per union-mask bit.
+@pytest.mark.parametrize("M,K,s,K_L", [(64, 1024, 0.5, 1024), (37, 300, 0.5, 256), (160, 2176, 0.7, 256), (48, 512, 1.0, 512)])
+def test_w2_round_trip_and_stats(b, M, K, s, K_L):
+    W = workloads.make_weight_w2(M, K, s, seed=M + K + 11)
+    assert W.min() >= -2 and W.max() <= 1
+    h = b.us_encode(W, fmt=(16, K_L, 2, 2), max_N=8, flags=b.US_ENCODE_HOST_ONLY | b.US_ENCODE_W2)
+    try:
+        assert (b.us_decode(h) == W).all()
+        st = b.us_get_stats(h)
+        ref = oracle.encode(W, 16, K_L, 2, 2)["stats"]     # same union mask; the oracle packs INT4 values
+        assert st["weight_bits"] == 2
+        assert st["nnz"] == ref["nnz"] and st["sum_P"] == ref["sum_P"] and st["n_tiles"] == ref["n_lt"]
+        assert st["bytes_payload"] == ref["sum_P"]         # Q * P_t values of 2 bits = P_t bytes
+        assert 2 * st["bytes_payload"] == ref["bytes_payload"]
+        assert st["bytes_bitmap"] == ref["bytes_bitmap"] and st["bytes_offsets"] == ref["bytes_offsets"]
+        # Eq. 1 with B_w = 0.25 bytes per weight
+        assert st["pmr"] == pytest.approx(0.25 * ref["nnz"] / (ref["bytes_bitmap"] + ref["bytes_offsets"]), rel=1e-12)
+        assert st["pmr"] == pytest.approx(0.5 * ref["pmr"], rel=1e-12)
+    finally:
+        b.us_destroy(h)
+
+
+def test_w2_errors(b):
+    W = np.zeros((16, 256), np.int8)
+    W[2, 3] = 2                                            # outside [-2, 1]
+    with pytest.raises(b.UsError) as e:
+        b.us_encode(W, fmt=(16, 256, 2, 2), flags=b.US_ENCODE_HOST_ONLY | b.US_ENCODE_W2)
+    assert e.value.status == 2
+    W[2, 3] = -2
+    for fmt in [(16, 256, 2, 1), (16, 64, 2, 2), None]:    # only the folded kernel layout holds INT2 weights
+        with pytest.raises(b.UsError) as e:
+            b.us_encode(W, fmt=fmt, flags=b.US_ENCODE_HOST_ONLY | b.US_ENCODE_W2)
+        assert e.value.status == 4, fmt
+    with pytest.raises(b.UsError) as e:
+        b.us_encode(W, fmt=(16, 256, 2, 2), flags=b.US_ENCODE_HOST_ONLY | b.US_ENCODE_W2 | b.US_ENCODE_PAIR_ROWS)
+    assert e.value.status == 4
+
+
 def test_pack_int4(b):
     X = np.array([[1, -2, 7, -8, 0]], np.int8)
     assert list(b.pack_int4(X)[0]) == [0x1 | (0xE << 4), 0x7 | (0x8 << 4), 0x0]

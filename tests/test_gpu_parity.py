@@ -411,3 +411,25 @@ def test_folded_format_limits(b):
         assert float(y.abs().max()) == 0.0
     finally:
         sw.close()
+
+
+# ---- W2A4: INT2 weights in the folded format, one payload byte per union-mask bit ----
+@pytest.mark.parametrize("M,K,s,K_L,Ns", [
+    (1024, 1024, 0.5, 256, [1, 8]), (1024, 1024, 0.5, 1024, [3, 8, 16]),
+    (2000, 1000, 0.5, 512, [5, 8, 24]),           # ragged rows and columns
+    (4096, 4096, 0.3, 512, [8]), (4096, 4096, 0.7, 512, [8, 32]),
+    (4096, 11008, 0.5, 1024, [8, 32, 64]),        # several K ranges / global split-K
+    (48, 512, 1.0, 512, [8]), (16, 256, 0.0, 256, [8]),
+])
+def test_w2a4(b, M, K, s, K_L, Ns):
+    seed = 680 + M % 91 + K % 83
+    W = workloads.make_weight_w2(M, K, s, seed=seed)
+    X = workloads.make_x(K, max(Ns), seed=seed)
+    s_w, s_x = workloads.make_scales(M, max(Ns), seed=seed)
+    _check_case(b, W, X, Ns, s_w, s_x, fmt=(16, K_L, 2, 2), flags=b.US_ENCODE_W2, max_N=max(Ns))
+
+
+def test_w2a4_70b_full_size(b):
+    W = workloads.make_weight_w2(28672, 8192, 0.6, seed=500)
+    X = workloads.make_x(8192, 8, seed=500)
+    _check_case(b, W, X, [8, 1], fmt=(16, 1024, 2, 2), flags=b.US_ENCODE_W2, max_N=8)
