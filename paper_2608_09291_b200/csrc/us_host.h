@@ -17,6 +17,14 @@
 //                 matrix sits in shared-memory bank l: every decode load is conflict free.
 //   * per-tile offsets: item_off[t] in units of 16 bytes, n_items + 1 entries.
 //
+// Folded variant (H_L = 16, R_A = 2, C_A = 2, Q = 4; K_L a multiple of 256): the tile's columns form two
+// areas of K_L/2; a mask bit covers rows g, g+8 at column k of BOTH areas, i.e. the same slot of k-blocks kb
+// and kb + K_L/64. The mask matrix has K_L/256 rows; a set bit owns one payload byte per area, at the same
+// position of two streams whose 128-byte rows alternate in the payload matrix ([2J rows][32 lanes]).
+// INT2 weights (w2, folded variant only): one stream; the byte of a set bit packs the bit's four 2-bit values,
+// each + 2 -- bits 1:0 = W[g][k], 3:2 = W[g+8][k] of area 0, bits 5:4 and 7:6 the same of area 1; a cleared
+// bit stands for 0xAA.
+//
 // Any other valid IE-BME format (other H_L, R_A, C_A, narrow tiles) is encoded on the host in the
 // paper's own array layout (GenericArrays) for us_get_stats / us_decode; no kernel reads it.
 #pragma once
@@ -43,7 +51,7 @@ struct HostMatrix {
     bool w2 = false;             // INT2 weights: one payload byte per union-mask bit of the (16, K_L, 2, 2) format
     GenericArrays gen;
     int32_t nkb = 0;        // k-blocks (32 columns) per tile
-    int32_t mask_rows = 0;  // nkb / 4
+    int32_t mask_rows = 0;  // mask words per lane and tile: nkb / (4 * C_A)
     int64_t n_strips = 0, n_segs = 0, n_items = 0;
     std::vector<int32_t> row_order;   // Mp entries: original row at padded position, -1 = padding
     std::vector<uint32_t> item_off;   // n_items + 1, units of 16 bytes

@@ -15,6 +15,9 @@
 //              one mask byte indexes a 256-entry selector table; two byte-permutes deposit the
 //              payload bytes of the lane's stream into the 8 fragment slots, absent positions
 //              take the neutral byte 0x08. All loads hit the lane's own shared-memory bank.
+//              Folded tiles (C_A = 2): one mask byte serves two k-blocks whose payload bytes sit at the
+//              same position of two streams; INT2 weights: one stream whose bytes are split into two
+//              nibbles after the gather (process_tile<.., CA, W2>).
 //   MMA        mma.sync m16n8k32 s8: fragment rows g carry the raw payload bytes
 //              (16*w_hi + (w_lo+8)), rows g+8 the low nibbles (w_lo+8); with Sx = sum_k x,
 //              Y_lo = E - 8*Sx and Y_hi = (RAW - E)/16, all exact in INT32.
