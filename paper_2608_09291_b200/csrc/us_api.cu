@@ -292,6 +292,9 @@ cudaError_t launch_st(const us::SpmmParams& p, bool xp, int grid, int block, int
         return timed ? cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NP, ST, true, true, true>, p)
                      : cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NP, ST, true, false, true>, p);
     }
+    if (NT == 1 && p.N == 1 && !timed)   // a single token: dp4a beats the MMA (measured 2-3 %)
+        return la ? cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<1, ST, true, false, false, false, 1, false, true>, p)
+                  : cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<1, ST, false, false, false, false, 1, false, true>, p);
     if (la && !timed) return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, ST, true, false>, p);
     if (!la && !timed) return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, ST, false, false>, p);
     if (la) return cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, ST, true, true>, p);
@@ -318,6 +321,10 @@ cudaError_t enable_large_smem_st(int bytes)
     if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, ST, false, false, false, true>, attr, bytes);
     constexpr int NP = NT <= 4 ? NT : 4;   // packed-X kernels exist for N <= 32
     if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NP, ST, true, false, true, true>, attr, bytes);
+    if (NT == 1) {   // single-token kernels
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<1, ST, true, false, false, false, 1, false, true>, attr, bytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<1, ST, false, false, false, false, 1, false, true>, attr, bytes);
+    }
     // folded tiles, INT4 and INT2
     if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, ST, true, false, false, false, 2, true>, attr, bytes);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(us::us_spmm_kernel<NT, ST, false, false, false, false, 2, true>, attr, bytes);

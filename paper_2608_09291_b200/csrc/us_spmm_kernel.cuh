@@ -429,7 +429,11 @@ __device__ __forceinline__ void store_rows(const StoreCtx p, const int (&v)[NT][
 // nibble = column area 0 (bits 1:0 row g, 3:2 row g + 8), high nibble = column area 1. One stream, gathered as
 // for CA = 1, then split: fragment rows g take the nibble 4 * (w_hi + 2) + (w_lo + 2), rows g + 8 its low two
 // bits w_lo + 2; with S = sum of x over the tile's columns, Y_lo = E - 2 S and Y_hi = (RAW - E) / 4 - 2 S.
-template <int NT, bool XP, int CA, bool W2 = false>
+// DP (N = 1 only; NT = 1, CA = 1, plain X): no MMA. xb_a then addresses token 0's activations at this lane's own
+// eight columns, and the lane accumulates its part of the two sums with four dp4a per k-block: c[0][0] = RAW,
+// c[0][2] = E. The caller adds the four lanes of a row group. Measured against the MMA at N = 1 (which wastes
+// seven of its eight token columns): 2-3 % faster on every shape.
+template <int NT, bool XP, int CA, bool W2 = false, bool DP = false>
 __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, uint32_t lut_stride,
                                              uint32_t xb_a, int xstride, int mask_rows, int lane,
                                              int (&c)[NT][4], uint32_t x_fold)
@@ -511,10 +515,16 @@ __device__ __forceinline__ void process_tile(uint32_t slot_a, uint32_t lut_a, ui
                 const uint32_t d0 = prmt(lo, kFill, e[i]);
                 const uint32_t d1 = prmt(prev, kFill, e[i] >> 16);
                 const uint32_t e0 = d0 & 0x0F0F0F0Fu, e1 = d1 & 0x0F0F0F0Fu;
+                if (DP) {
+                    const uint2 b = kPreX ? xf[i][0] : ldx(xb_a + kXStep * (4 * w + i));
+                    c[0][0] = __dp4a((int)d0, (int)b.x, c[0][0]); c[0][0] = __dp4a((int)d1, (int)b.y, c[0][0]);
+                    c[0][2] = __dp4a((int)e0, (int)b.x, c[0][2]); c[0][2] = __dp4a((int)e1, (int)b.y, c[0][2]);
+                } else {
 #pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
-                    const uint2 b = kPreX ? xf[i][nt] : ldx((ca ? xb_fold_a : xb_a) + kXStep * (4 * w + i) + nt * 8 * xstride);
-                    mma_s8(c[nt], d0, e0, d1, e1, b.x, b.y);
+                    for (int nt = 0; nt < NT; ++nt) {
+                        const uint2 b = kPreX ? xf[i][nt] : ldx((ca ? xb_fold_a : xb_a) + kXStep * (4 * w + i) + nt * 8 * xstride);
+                        mma_s8(c[nt], d0, e0, d1, e1, b.x, b.y);
+                    }
                 }
             }
             }
@@ -564,8 +574,9 @@ constexpr int kTimerWords = kWarpRec * kMaxWarpsPerCta * kMaxCtas;
 // AM = chained call that leaves the per-token absmax of its fp16 output (separate too: the plain
 // fp16 store measured 2.5 % slower with the tracking compiled in behind a run-time flag).
 // CA = column areas of the weight format (2: folded tiles).
-// W2 = INT2 weights (folded format only).
-template <int NT, int STAGES, bool LA, bool TIMED, bool XP = false, bool AM = false, int CA = 1, bool W2 = false>
+// W2 = INT2 weights (folded format only). DP = dp4a instead of the MMA: the N = 1 kernels of the default format.
+template <int NT, int STAGES, bool LA, bool TIMED, bool XP = false, bool AM = false, int CA = 1, bool W2 = false,
+          bool DP = false>
 // (N <= 8 kernels are compiled for up to 20 warps: 80 registers instead of 90, which lets 12 instead of 10 warps of
 // two half-SM CTAs share an SM; more than 16 warps per full-SM CTA were measured and do not pay.)
 __global__ void __launch_bounds__((NT == 1 && CA == 1) ? 640 : 512, 1) us_spmm_kernel(const SpmmParams p)
@@ -965,8 +976,20 @@ __global__ void __launch_bounds__((NT == 1 && CA == 1) ? 640 : 512, 1) us_spmm_k
             const uint32_t slot_a = smem_u32(my_ring + (size_t)cur * p.slot_bytes);
             const uint32_t xb_a = XP ? smem_u32(x8) + (lane >> 2) * xstride + 4 * (lane & 3) + sgl * (p.K_L / 2)
                                      : smem_u32(x8) + (lane >> 2) * xstride + 8 * (lane & 3) + sgl * p.K_L;
-            process_tile<NT, XP, CA, W2>(slot_a, lut_a, 4u * (uint32_t)p.lut_rep, xb_a, xstride, p.mask_rows, lane, c,
-                                     (uint32_t)p.fold_kb * (XP ? 16u : 32u));
+            if (DP) {
+                const uint32_t xb0 = smem_u32(x8) + 8 * (lane & 3) + sgl * p.K_L;   // token 0, this lane's columns
+                process_tile<NT, XP, CA, W2, true>(slot_a, lut_a, 4u * (uint32_t)p.lut_rep, xb0, xstride, p.mask_rows, lane, c, 0u);
+                // the four lanes of a row group hold parts of the same two sums; the first keeps them in the
+                // accumulator slots of token 0, the slots of tokens 1..7 stay zero
+                int r = c[0][0], e = c[0][2];
+                r += __shfl_xor_sync(0xffffffffu, r, 1); r += __shfl_xor_sync(0xffffffffu, r, 2);
+                e += __shfl_xor_sync(0xffffffffu, e, 1); e += __shfl_xor_sync(0xffffffffu, e, 2);
+                const bool first = (lane & 3) == 0;
+                c[0][0] = first ? r : 0; c[0][2] = first ? e : 0;
+            } else {
+                process_tile<NT, XP, CA, W2>(slot_a, lut_a, 4u * (uint32_t)p.lut_rep, xb_a, xstride, p.mask_rows, lane, c,
+                                             (uint32_t)p.fold_kb * (XP ? 16u : 32u));
+            }
             __syncwarp();
             const long long t2c = timing ? clock64() : 0;
 
