@@ -427,6 +427,9 @@ us_status enqueue_spmm(us_handle* h, const void* X, int32_t N, const void* x_sca
         const int64_t per_cta = std::max<int64_t>(1, hm.n_items / std::max(1, h->sm_count));
         const int balanced = (int)std::max<int64_t>(1, per_cta / (4 * (int64_t)g.warps));
         p.run_len = std::max(1, std::min(std::min(p.G, 2 * balanced), p.G));
+        // Fewer tiles than warps: one tile per warp, all at once (1024 x 1024, N = 8: 4.1 -> 3.1 us); with more
+        // tiles than warps, runs of two keep a run's sums in registers and win (4096 x 4096: 5.7 against 6.3 us).
+        if ((hm.n_items + h->sm_count - 1) / std::max(1, h->sm_count) <= g.warps) p.run_len = 1;
     }
     p.row_order = h->d_row_order; p.w_scale = h->d_w_scale;
     p.X = static_cast<const uint8_t*>(X);
