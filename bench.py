@@ -36,8 +36,8 @@ METRIC = "w4a4_spmm_achieved_hbm_gbs"
 UNIT = "GB/s"
 HEAD = dict(M=4096, K=4096, s=0.5, N=8, seed=201)
 WORKLOAD = ("llama2-7b attention projection 4096x4096 INT4, 50% uniform sparsity, N=8, fused fp16 dequant; "
-            "bytes counted at local tiles of 16x512, one union-mask bit per 2x1 values")
-HEAD_K_L = 512                       # tile width the byte count of both arms refers to
+            "bytes counted at local tiles of 16x1024, one union-mask bit per 2x1 values")
+HEAD_K_L = 1024                       # tile width the byte count of both arms refers to
 CONTRACT_PEAK_GBS = 8000.0
 L2_BYTES_FALLBACK = 126 * 1024 * 1024
 MIN_TIMED_SECONDS = 0.5

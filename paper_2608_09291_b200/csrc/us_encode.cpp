@@ -107,12 +107,15 @@ void pair_rows(const int8_t* W, int64_t M, int64_t K, int threads, HostMatrix* h
 
 int32_t default_K_L(int64_t M, int64_t K, int n_sm)
 {
-    // Large tiles keep the per-tile padding of the lane streams small; small matrices get
-    // smaller tiles so that every warp of every SM still finds work.
-    // (Measured on a 4096 x 4096 matrix at 50 % sparsity: 512 beats both 256 and 1024.)
+    // Large tiles keep the per-tile padding of the lane streams and the per-tile bookkeeping small; small
+    // matrices get smaller tiles so that every warp of every SM still finds work. From about four tiles of
+    // 1024 columns per SM on, 1024 wins: a CTA then has no more tiles than warps, each warp decodes one tile
+    // and nothing waits for a second round of copies (measured at 50 % sparsity, N = 8, K_L = 256 / 512 / 1024 /
+    // 2048: 4096 x 4096 6.7 / 5.7 / 4.8 / 6.3 us, 5120 x 5120 at N = 16 10.8 / 9.1 / 8.4 / 9.8, 11008 x 4096
+    // 11.9 / 10.9 / 9.0 / 8.8; 2048 x 2048 3.7 / 3.8 / 4.2 / 5.2, 1024 x 1024 3.1 / 3.4 / 3.6 / 4.5).
     const int64_t strips = (M + 15) / 16;
     if (n_sm <= 0) n_sm = 148;
-    if (strips * ((K + 1023) / 1024) >= (int64_t)n_sm * 16) return 1024;
+    if (strips * ((K + 1023) / 1024) >= (int64_t)n_sm * 4) return 1024;
     if (strips * ((K + 511) / 512) >= (int64_t)n_sm * 4) return 512;
     return 256;
 }
