@@ -171,7 +171,7 @@ def test_layer_13b_chain(b, j, s):
                 ref = oracle.spmm_dense(m["W"], q)
                 assert np.isfinite(got).all() and np.abs(got).max() > 0
                 ok = oracle.fp16_within_tolerance(got, ref, m["s_w"], st, rel=2e-3)
-                assert ok.all(), f"round {rnd}: {int((~ok).sum())} outputs outside tolerance"
+                assert ok.all(), f"pass {rnd}: {int((~ok).sum())} outputs outside tolerance"
                 m0, m1 = m["rng"]
                 assert np.array_equal(b.amax_values(m["amax"], N), _amax_words(oracle.absmax_f16(got, m0, m1)))
                 prev = got[:, m0:m1]
