@@ -656,8 +656,11 @@ __global__ void __launch_bounds__((NT == 1 && CA == 1) ? 640 : 512, 1) us_spmm_k
     };
     uint32_t run_next = 0, run_end = 0;   // the run being handed out (after the fixed positions)
     int static_k = STAGES + 1;            // fixed positions already handed out
+    // (a CTA whose fixed positions already cover its whole range never touches the counter)
+    const bool all_static = beg + (uint32_t)n_static * (uint32_t)n_warps * R >= end;
     auto next_pos = [&]() -> uint32_t {
         if (static_k < n_static * (int)R) return static_pos(static_k++);
+        if (all_static) return end;
         if (run_next == run_end) {
             // Guided chunks: as long as every warp can still get a run of R (a whole strip's
             // segments when R = G: its sums never leave the registers), hand out R; towards the end
