@@ -493,8 +493,8 @@ def kernel_label(binding, handle, N):
 
 # Measured DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch, from the ncu
 # captures of the same kernel build (one launch each; commands in the capture summaries).
-TRAFFIC_BYTES_PER_LAUNCH = 7_968_768          # 4096x4096, s = 0.5, N = 8, fp16: 7.9688 MB read, 0 written
-TRAFFIC_BYTES_PER_LAUNCH_LARGE = 101_139_968  # 28672x8192, s = 0.6, N = 8, int32: 98.01 MB read + 3.13 MB written
+TRAFFIC_BYTES_PER_LAUNCH = 7_969_024          # 4096x4096, s = 0.5, N = 8, fp16: 7.9690 MB read, 0 written
+TRAFFIC_BYTES_PER_LAUNCH_LARGE = 101_235_968  # 28672x8192, s = 0.6, N = 8, int32: 98.02 MB read + 3.22 MB written
 
 
 def sweep(binding, torch, workloads, l2, peak_gbs):
