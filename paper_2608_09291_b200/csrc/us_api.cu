@@ -64,6 +64,7 @@ constexpr int kLocalAccBudget = 32 * 1024;   // local strip sums a K-range width
 constexpr int kLocalAccCap = 48 * 1024;      // ... and what is taken if nothing fits that
 constexpr int kMinWarps = 12;                // warps the automatic K-range choice keeps room for
 constexpr int kCoresidentTiles = 16;         // most tiles per CTA for the half-SM plan
+constexpr int kHalfSmBytes = 228 * 1024 / 2 - 1024 - 512;   // shared memory of a half-SM CTA: 228 KB per SM, 1 KB reserved per CTA
 
 struct LaunchGeom {
     int nt, cls, warps, stages, smem, lut_rep;
@@ -159,7 +160,7 @@ bool plan_launch(const us_handle* h, int N, LaunchGeom* g)
     // (Tried at N = 32 as well: 8 warps per CTA, slower.)
     const bool co_class = g->nt == 1 || (g->nt == 2 && g->xp && s_local > 0);
     if (coresident_knob() && co_class && per_cta <= kCoresidentTiles && stages_knob() == 0) {
-        const int half = 228 * 1024 / 2 - 1024 - 512;   // per SM: 228 KB, 1 KB reserved per CTA
+        const int half = kHalfSmBytes;
         const int fixed8 = fixed_for(8) + 32 * 8;
         const bool fold = h->host.fmt.C_A == 2;
         int w = std::min(g->nt == 1 ? (fold ? h->co_warps_fold : h->co_warps) : h->co_warps2,
@@ -229,7 +230,24 @@ void plan_classes(us_handle* h, int n_cta, std::vector<uint32_t> (&sched)[4])
             const int64_t n_segs = h->host.n_segs;
             const int64_t ranges = h->s_local[c] > 0 ? (n_segs + h->G[c] - 1) / h->G[c] : n_segs + 1;
             const bool small_share = nt >= 2 && (int64_t)h->host.blob.size() / std::max(1, n_cta) < 128 * 1024;
-            if (ranges > 1 || small_share) {
+            // N <= 8: packed X when that is what lets the half-SM plan of plan_launch hold its eight warps
+            // (4096 x 4096 at 30 % sparsity: tiles of 9.5 KB and 32 KB of int8 X do not fit half an SM, with
+            // 16 KB of packed X they do: 5.6 -> 4.6 us; the same for the folded format at 50 %: 5.3 -> 4.35)
+            bool for_half_sm = false;
+            if (nt == 1 && ranges == 1 && coresident_knob()) {
+                const int64_t per_cta = (h->host.n_items + n_cta - 1) / std::max(1, n_cta);
+                const int64_t need = 8;
+                auto fits = [&](bool xp, int s_loc) {
+                    const int64_t fixed8 = 256 * 8 * 4 + (int64_t)us::kLutScratchBytes + x_bytes(nt, n_segs, h->host.fmt.K_L, xp) +
+                                           n_segs * nt * 8 * 4 + us::kClaimWords * 4 + (int64_t)s_loc * (nt * 128 + 1) * 4 +
+                                           2 * us::kOffTable * 4 + 128 + 32 * 8;
+                    return fixed8 + need * (int64_t)slot_bytes_for(h->host) <= kHalfSmBytes;
+                };
+                // (only where every tile then finds its own warp: 5120 x 5120 at 70 % sparsity, 11 tiles per CTA,
+                // runs 7.7 us in a 12-warp half-SM CTA against 6.3 us with 16 warps on the whole SM)
+                for_half_sm = per_cta <= 8 && !fits(false, h->s_local[c]) && fits(true, h->s_local[c]);
+            }
+            if (ranges > 1 || small_share || for_half_sm) {
                 std::vector<uint32_t> alt;
                 int sl2 = 0;
                 const int G2 = local_plan(true, &alt, &sl2);
@@ -271,7 +289,7 @@ cudaError_t launch_st(const us::SpmmParams& p, bool xp, int grid, int block, int
         return la ? cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, ST, true, false, false, false, 2, true>, p)
                   : cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<NT, ST, false, false, false, false, 2, true>, p);
     if (p.fold_kb) {   // folded tiles (two column areas); stage timers for the N <= 8 kernels only
-        if (NT == 1 && timed)
+        if (NT == 1 && timed && !xp)
             return la ? cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<1, ST, true, true, false, false, 2>, p)
                       : cudaLaunchKernelEx(&cfg, us::us_spmm_kernel<1, ST, false, true, false, false, 2>, p);
         if (NT <= 4 && xp && la) {
@@ -437,8 +455,9 @@ us_status enqueue_spmm(us_handle* h, const void* X, int32_t N, const void* x_sca
     p.X = static_cast<const uint8_t*>(X);
     p.x_scale = static_cast<const uint16_t*>(x_scale);
     p.Y = Y; p.acc = acc; p.cnt = cnt; p.err = h->d_err;
-    // (no stage-timer builds of the absmax-tracking kernels, nor of the folded-tile kernels for N > 8)
-    p.timers = (timers && !(chain && chain->y_amax) && !(hm.fmt.C_A == 2 && g.nt > 1) && !hm.w2) ? h->d_timers : nullptr;
+    // (no stage-timer builds of the absmax-tracking kernels, nor of the folded-tile kernels for N > 8 or with packed X:
+    // a timer build launched on a plan laid out for another variant would index shared memory wrongly)
+    p.timers = (timers && !(chain && chain->y_amax) && !(hm.fmt.C_A == 2 && (g.nt > 1 || g.xp)) && !hm.w2) ? h->d_timers : nullptr;
     p.M = (int32_t)hm.M; p.K = (int32_t)hm.K; p.N = N;
     p.n_strips = (int32_t)hm.n_strips; p.n_segs = (int32_t)hm.n_segs;
     p.mask_rows = hm.mask_rows; p.K_L = hm.fmt.K_L;

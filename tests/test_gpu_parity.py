@@ -433,3 +433,30 @@ def test_w2a4_70b_full_size(b):
     W = workloads.make_weight_w2(28672, 8192, 0.6, seed=500)
     X = workloads.make_x(8192, 8, seed=500)
     _check_case(b, W, X, [8, 1], fmt=(16, 1024, 2, 2), flags=b.US_ENCODE_W2, max_N=8)
+
+
+def test_stage_timers_on_every_plan_variant(b):
+    """Switching the stage timers on must never launch a kernel variant the plan was not laid out for: plans
+    without a timer build (folded tiles with packed activations, INT2 weights, N > 8 on folded tiles) simply
+    run untimed. Values are checked with the timers on."""
+    cases = [((16, 1024, 2, 2), 0, 4096, 4096, 0.5, 8),      # folded, packed X (half-SM plan)
+             ((16, 1024, 2, 2), 0, 1024, 2048, 0.5, 16),     # folded, N > 8
+             ((16, 512, 2, 2), b.US_ENCODE_W2, 1024, 1024, 0.5, 8),
+             ((16, 1024, 2, 1), 0, 4096, 4096, 0.3, 8),      # default format, packed X (half-SM plan)
+             (None, 0, 1024, 1024, 0.5, 8)]
+    for fmt, flags, M, K, s, N in cases:
+        W = workloads.make_weight_w2(M, K, s, seed=77) if flags & b.US_ENCODE_W2 else workloads.make_weight(M, K, s, seed=77)
+        X = workloads.make_x(K, N, seed=77)
+        sw = b.SparseWeight(W, None, fmt=fmt, max_N=N, flags=flags)
+        try:
+            b.us_stage_timers(sw.handle, 1)
+            Xd = torch.from_numpy(b.pack_int4(X)).cuda()
+            for _ in range(2):
+                y = sw.spmm(Xd, N)
+                torch.cuda.synchronize()
+                sw.check()
+                assert (y.cpu().numpy() == oracle.spmm_dense(W, X)).all(), (fmt, flags, M, K, N)
+            d = b.us_stage_timers(sw.handle, 0, read=True)
+            assert d["warps"] >= 0
+        finally:
+            sw.close()
